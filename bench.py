@@ -1,0 +1,394 @@
+"""Benchmark of the hooked paged-attention path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one pass of the whole hot path (page resolve, scores, online softmax, span masses, PV,
+steering add, store and -- for decode -- the split-K merge) over one batch of seeded synthetic
+input.  The default workload is the decode batch (64 sequences, contexts 512..4096, 32/8 heads,
+head_dim 128, 16 probed heads, 2 spans, 4 steered heads); `--workload` selects the others.
+
+The printed JSON line carries the whole-job throughput with inputs resident in HBM (`value`), the
+same metric through the public call with host buffers (`e2e`), the roofline of the dominant kernel,
+the hook overhead against the same kernels with hooks disabled, and the fp64 CPU oracle timed on
+the host cores (`cpu_baseline`; a reported baseline, not the target).
+
+With N > 1 (torchrun) every rank runs an independent replica of the workload -- the path has no
+exchange step, so there is no collective on the data path; timing is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2603_06588_b200 import inputs  # noqa: E402
+
+METRIC = "hooked-attn tokens/s"
+UNIT = "tokens/s"
+
+WORKLOADS = {
+    "cfg2_decode": "decode batch: 64 seqs x 1 token, ctx U[512,4096], Hq32/Hkv8, D128, 16 probed heads, 2 spans, 4 steered heads",
+    "cfg3_prefill": "prefill: 8 seqs x 4096 tokens causal, Hq32/Hkv8, D128, ~10% (layer,head) pairs probed, 3 spans, one layer call per step",
+    "cfg4_decode": "mixed batch, decode part: 256 seqs, ctx U[1024,8192], Hq28/Hkv4, D128, 14 probed heads, 4 spans, 8 steered heads",
+    "cfg4_prefill": "mixed batch, prefill part: 2 chunks of 2048 tokens on 4096-token contexts, Hq28/Hkv4, D128",
+    "cfg5_decode": "long context decode: 4 seqs at 32768+ keys, Hq64/Hkv8, D128, 64 probed heads, 8 spans, 8 steered heads",
+    "cfg5_prefill": "long context prefill: 4 seqs x 32768 tokens causal, Hq64/Hkv8, D128, 64 probed heads, 8 spans, 8 steered heads",
+}
+
+
+def make_workload(name: str):
+    if name == "cfg2_decode":
+        return inputs.config2_decode()
+    if name == "cfg3_prefill":
+        return inputs.config3_prefill(layer=0, force_probe=True)
+    if name == "cfg4_decode":
+        return inputs.config4_decode()
+    if name == "cfg4_prefill":
+        return inputs.config4_prefill()
+    if name == "cfg5_decode":
+        return inputs.config5_decode(step=64)
+    if name == "cfg5_prefill":
+        return inputs.config5_prefill()
+    raise SystemExit(f"unknown workload {name}; choose from {sorted(WORKLOADS)}")
+
+
+def algorithmic_work(case):
+    """Algorithmic bytes and flops of one step: every needed K and V element once per KV head,
+    plus q, out, span_mass and the tables; flops = 4*D per visible (row, key, query head)."""
+    D, Hq, Hkv = case.head_dim, case.num_q_heads, case.num_kv_heads
+    kv_bytes = case.kv_tokens() * Hkv * D * 2 * 2
+    qo_bytes = 2 * case.total_q * Hq * D * 2
+    rows = case.num_seqs if (case.is_decode or case.probe_rows == inputs.PROBE_ROWS_LAST) else case.total_q
+    misc = rows * case.num_probed * case.num_spans * 4 + case.kv_tokens() // inputs.PAGE * 4 + case.num_seqs * 8
+    flops = 4.0 * D * case.visible_pairs() * Hq
+    return kv_bytes + qo_bytes + misc, flops
+
+
+# ------------------------------------------------------------------------------------------------
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            m = json.load(f)
+        return {"hbm_gbs": float(m["hbm_gbs"]), "bf16_tflops": float(m["bf16_tflops"]),
+                "bf16_tflops_sustained": float(m.get("bf16_tflops_sustained", m["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.file.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            # samples under load: the upper half of the observed clocks (idle samples sit low)
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The oracle, as it stands, timed on the host cores on the same workload and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle
+    case = make_workload(args.workload)
+    # every step is a bounded sample, sized so that the whole run ends within a few minutes
+    budget = min(args.ref_budget, 120.0 / max(1, args.steps + args.warmup))
+    rows, desc, scale_tokens = oracle_sample(case, budget_s=budget)
+    for _ in range(args.warmup):
+        oracle.run(case, rows=rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.run(case, rows=rows)
+    dt = (time.perf_counter() - t0) / args.steps
+    tokens = scale_tokens
+    val = tokens / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def oracle_sample(case, budget_s: float):
+    """A bounded sample of the workload for the CPU oracle: global query rows, a description, and
+    the number of tokens the timing is scaled to (rows evaluated, weighted by visible keys so that
+    the figure stays a tokens/s of the same workload)."""
+    total_pairs = case.visible_pairs()
+    # the oracle sustains roughly 3e8 (key, d) multiply-adds per core-second; size by that
+    macs_per_row_key = 2 * case.head_dim * case.num_q_heads
+    budget_pairs = budget_s * 2.5e9 / macs_per_row_key
+    if total_pairs <= budget_pairs:
+        return None if False else list(range(case.total_q)), f"all {case.total_q} query rows x {case.num_q_heads} heads", case.total_q
+    rows = inputs.sample_rows(case, extra_random=0)
+    cu = case.cu_q_lens.tolist()
+    Ls = case.seq_lens.tolist()
+    picked, pairs = [], 0
+    stride = max(1, len(rows) // 64)
+    for r in rows[::stride]:
+        s = max(i for i in range(case.num_seqs) if cu[i] <= r)
+        pos = Ls[s] - (cu[s + 1] - cu[s]) + (r - cu[s])
+        if pairs + pos + 1 > budget_pairs and picked:
+            break
+        picked.append(r)
+        pairs += pos + 1
+    tokens = case.total_q * pairs / total_pairs
+    return picked, (f"{len(picked)} sampled query rows x {case.num_q_heads} heads ({pairs} of {total_pairs} visible pairs per head); "
+                    "tokens/s extrapolated by visible-pair count"), tokens
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", default="cfg2_decode")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-budget", type=float, default=2.0, help="seconds of CPU time per oracle step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.workload not in WORKLOADS:
+        raise SystemExit(f"unknown workload {args.workload}; choose from {sorted(WORKLOADS)}")
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    from paper_2603_06588_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = world > 1
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    if dist:
+        import torch.distributed as td
+        td.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist:
+            td.barrier()
+        torch.cuda.synchronize()
+
+    case = make_workload(args.workload)
+    eng = binding.HookAttn(local)
+    kw = binding.case_to_device(case, f"cuda:{local}")
+    kw_off = binding.case_to_device(case.without_hooks(), f"cuda:{local}")
+    for k in ("q", "k_cache", "v_cache", "block_table", "seq_lens", "cu_q_lens"):
+        if k in kw:
+            kw_off[k] = kw[k]                       # same device tensors, hooks disabled
+    status = torch.zeros(1, dtype=torch.int32, device=f"cuda:{local}")
+    plan_hook = eng.plan(case.is_decode, status=status, **kw)      # marshals once, allocates outputs
+    plan_off = eng.plan(case.is_decode, **kw_off)
+    plan_hook.run()
+    plan_off.run()
+    out, mass = plan_hook.out, plan_hook.span_mass
+    torch.cuda.synchronize()
+    if int(status.item()) != 0:
+        raise SystemExit(f"device status {binding.strerror(int(status.item()))}")
+    launches_per_step = 2 if case.is_decode else 1
+
+    def timed(n, plan):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record()
+        for _ in range(n):
+            plan.run()
+        ev1.record()
+        barrier()
+        return ev0.elapsed_time(ev1) / 1e3
+
+    alg_bytes, alg_flops = algorithmic_work(case)
+    working_set_mb = alg_bytes / 1e6
+    flush = None
+    if working_set_mb < 256:                         # inputs do not exceed L2: flush between iterations
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=f"cuda:{local}")
+
+    def timed_flushed(n, plan):
+        tot = 0.0
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        for _ in range(n):
+            flush.zero_()
+            ev0.record()
+            plan.run()
+            ev1.record()
+            ev1.synchronize()
+            tot += ev0.elapsed_time(ev1) / 1e3
+        barrier()
+        return tot
+
+    run_timed = timed if flush is None else timed_flushed
+    hooked, plain = plan_hook, plan_off
+
+    run_timed(args.warmup, hooked)
+    sampler = ClockSampler(local)
+    sampler.start()
+    t_hook = run_timed(args.steps, hooked)
+    clocks_timed = sampler.stop()
+
+    # hook overhead: same kernels with hooks disabled, interleaved with hooked passes
+    sampler2 = ClockSampler(local)
+    sampler2.start()
+    reps = 5
+    n_ov = max(10, args.steps // reps)
+    th, tp = [], []
+    for _ in range(reps):
+        tp.append(run_timed(n_ov, plain) / n_ov)
+        th.append(run_timed(n_ov, hooked) / n_ov)
+    overhead = statistics.median(th) / statistics.median(tp) - 1.0
+
+    # end to end through the public call with host buffers: the step's inputs (queries, tables,
+    # lengths, spans) come from pinned host memory and the results go back to the host every step;
+    # the KV cache is state that stays resident on the device, like it does while serving.
+    host_in = {k: kw[k].cpu().pin_memory() for k in ("q", "block_table", "seq_lens", "cu_q_lens", "spans") if k in kw}
+    dev_in = {k: torch.empty_like(kw[k]) for k in host_in}
+    host_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    host_mass = None if mass is None else torch.empty(mass.shape, dtype=mass.dtype).pin_memory()
+    e2e_kw = dict(kw)
+    e2e_kw.update(dev_in)
+    plan_e2e = eng.plan(case.is_decode, out=out, span_mass=mass, **e2e_kw)
+    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
+    d2h = host_out.numel() * host_out.element_size() + (0 if host_mass is None else host_mass.numel() * 4)
+
+    def e2e_step():
+        for k, t in host_in.items():
+            dev_in[k].copy_(t, non_blocking=True)
+        plan_e2e.run()
+        host_out.copy_(out, non_blocking=True)
+        if host_mass is not None:
+            host_mass.copy_(mass, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    n_e2e = max(10, min(args.steps, 500))
+    for _ in range(3):
+        e2e_step()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(n_e2e):
+        e2e_step()
+    ev1.record()
+    barrier()
+    t_e2e = ev0.elapsed_time(ev1) / 1e3 / n_e2e
+    clocks_all = sampler2.stop()
+
+    if dist:
+        t = torch.tensor([t_hook, t_e2e], dtype=torch.float64, device=f"cuda:{local}")
+        td.all_reduce(t, op=td.ReduceOp.MAX)
+        t_hook, t_e2e = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peaks = load_peaks()
+        per_step = t_hook / args.steps
+        tokens = case.total_q
+        bound = "hbm" if case.is_decode else "tensor"
+        if bound == "hbm":
+            achieved = alg_bytes / per_step / 1e9
+            peak, unit = peaks["hbm_gbs"], "GB/s"
+        else:
+            achieved = alg_flops / per_step / 1e12
+            peak, unit = (peaks["bf16_tflops"] if t_hook < 2.0 else peaks["bf16_tflops_sustained"]), "TFLOP/s"
+        clocks = clocks_timed if clocks_timed["samples"] >= 3 else clocks_all
+        line = {
+            "metric": METRIC, "value": world * tokens / per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}",
+                       "l2": ("inputs larger than L2 (%.0f MB per step)" % working_set_mb) if flush is None
+                       else "L2 flushed between iterations (256 MB write)",
+                       "replicas": world, "kv_cache": "resident in HBM (state, not a per-step input)"},
+            "roofline": {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+                         "traffic": None, "peak_source": f"of {peaks['source']}",
+                         "kernel": "decode_splitk_kernel (+ decode_merge_kernel; duration = whole step, conservative)"
+                         if case.is_decode else "prefill kernel (one launch per step)",
+                         "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
+                         "frac_of_datasheet": achieved / (8000.0 if bound == "hbm" else 2250.0)},
+            "hook_overhead": overhead,
+            "ms_per_step_hooks_off": statistics.median(tp) * 1e3,
+            "e2e": {"value": world * tokens / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": t_e2e * 1e3},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                       "samples": clocks["samples"]},
+        }
+        if not args.no_cpu_baseline:
+            from oracle import oracle
+            rows, desc, scale_tokens = oracle_sample(case, budget_s=2.0)
+            oracle.run(case, rows=rows[: max(1, len(rows) // 8)])
+            t0 = time.perf_counter()
+            reps_cpu = 3
+            for _ in range(reps_cpu):
+                oracle.run(case, rows=rows)
+            dt = (time.perf_counter() - t0) / reps_cpu
+            line["cpu_baseline"] = {"value": scale_tokens / dt, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+                                    "sample": desc, "seconds_per_pass": dt}
+        print(json.dumps(line))
+    if dist:
+        td.barrier()
+        td.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

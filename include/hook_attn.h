@@ -1,0 +1,140 @@
+/*
+ * hook_attn.h -- C ABI of the hooked paged-attention library for NVIDIA B200 (sm_100a).
+ *
+ * One call computes, for a batch of sequences whose keys/values live in a paged KV cache,
+ *
+ *   (1) causal grouped-query attention   out[i,h,:] = softmax_t(scale * q[i,h,:].K[t,kv(h),:]) . V[t,kv(h),:]
+ *   (2) the passive probe: for every *probed* query head and every configured key span
+ *       [a_j, b_j) the exact post-softmax attention mass the query row places on the span,
+ *           span_mass[i,h,j] = sum_{t in [a_j,b_j), t <= pos(i)} p[i,h,t]
+ *       -- the quantity the paper's analyzer re-assembles from saved queries and keys and
+ *       aggregates over token ranges (Section 2.2, the AttntrackerAnalyzer listing:
+ *       "compute_attention_from_qk" followed by "attn2score" over "input_range"); the
+ *       probed heads are the config's "important_heads" of one layer (Section 2, config
+ *       listing), the probed rows its "hookq_mode" (last_token / all_tokens);
+ *   (3) the active intervention: out[i,h,:] += alpha[h] * steer_vec[h,:] on the steered
+ *       heads -- activation steering (Section 1, "Model Steering"; Section 3), applied per
+ *       attention head after the softmax normalisation and before the single rounding of
+ *       the output to bf16.
+ *
+ * Probing never changes `out` ("keeping the model generation intact", Section 1): with and
+ * without probes the output bits are identical.  No attention matrix is materialised and no
+ * query/key tensor leaves the GPU; span masses are carried as extra online-softmax
+ * accumulators.
+ *
+ * Geometry.  Sequence s has L_s = seq_lens[s] keys in the cache (INCLUDING the keys of the
+ * rows in this call: their K/V must already be written) and n_s query rows in this call.
+ * Row i of sequence s sits at absolute position pos = L_s - n_s + i and sees keys 0..pos.
+ * Logical key t of sequence s lives in physical page block_table[s][t / page_size], slot
+ * t % page_size.  Query head h reads KV head h / (num_q_heads / num_kv_heads).
+ *
+ * Pointers.  Unless a field says "host", every pointer is a DEVICE pointer owned by the
+ * caller and borrowed until the work enqueued by the call has completed on the stream.  The
+ * library writes only `out`, `span_mass`, `workspace` and `status`.  Calls enqueue work on the
+ * caller's stream, never synchronise, and never allocate device memory.  Return codes are
+ * synchronous and cover argument validation and launch errors; faults the device detects
+ * (a block-table entry outside [0, num_blocks), a sequence longer than its table, more rows
+ * than keys) are reported through the optional `status` word, the affected rows are written
+ * as zeros, and no out-of-range address is dereferenced.
+ *
+ * Supported: head_dim in {64, 128}; page_size = 16; num_q_heads % num_kv_heads == 0 with a
+ * group size <= 8; num_q_heads <= 64; num_spans <= 8; strides multiples of 8 elements and
+ * 16-byte aligned base pointers.  Anything else returns HOOK_ATTN_ERR_UNSUPPORTED.
+ */
+#ifndef HOOK_ATTN_H_
+#define HOOK_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hook_attn_handle hook_attn_handle; /* per-device state: SM count, cached descriptors */
+
+enum {
+    HOOK_ATTN_OK = 0,
+    HOOK_ATTN_ERR_INVALID_ARG = -1, /* null required pointer, negative size, inconsistent shapes */
+    HOOK_ATTN_ERR_UNSUPPORTED = -2, /* shape outside the supported set listed above */
+    HOOK_ATTN_ERR_WORKSPACE = -3,   /* workspace missing or smaller than hook_attn_workspace_bytes */
+    HOOK_ATTN_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (launch, attribute) */
+    HOOK_ATTN_ERR_TIMEOUT = -5,     /* device status: a bounded wait inside a kernel ran out */
+    HOOK_ATTN_ERR_BOUNDS = -6       /* device status: block id / length outside its range */
+};
+
+/* Which query rows of a prefill call are probed: the config's "hookq_mode" (Section 2). */
+enum {
+    HOOK_PROBE_ROWS_ALL = 0,  /* "all_tokens": span_mass has one row per query row */
+    HOOK_PROBE_ROWS_LAST = 1  /* "last_token": one row per sequence (its last query row) */
+};
+
+typedef struct {
+    /* ---- shapes ---- */
+    int32_t num_seqs;            /* sequences in the batch (>= 0) */
+    int32_t total_q;             /* total query rows T = sum n_s (decode: == num_seqs) */
+    int32_t num_q_heads;         /* Hq */
+    int32_t num_kv_heads;        /* Hkv */
+    int32_t head_dim;            /* D */
+    int32_t page_size;           /* tokens per KV page */
+    int32_t num_blocks;          /* physical pages in the cache (bounds for block_table) */
+    int32_t max_blocks_per_seq;  /* row length of block_table */
+    int32_t num_spans;           /* S spans per sequence (0 = no probe) */
+    int32_t probe_rows;          /* HOOK_PROBE_ROWS_*; ignored by decode (always LAST) */
+    float   scale;               /* softmax scale; <= 0 selects 1/sqrt(head_dim) */
+    int32_t reserved0;
+
+    /* ---- device tensors ---- */
+    const void*    q;            /* bf16 [total_q][Hq][D], contiguous */
+    const void*    k_cache;      /* bf16, element (block, slot, kv_head, d) at
+                                    block*kv_block_stride + slot*kv_token_stride + kv_head*kv_head_stride + d */
+    const void*    v_cache;      /* same layout and strides as k_cache */
+    int64_t        kv_block_stride, kv_token_stride, kv_head_stride; /* in elements */
+    const int32_t* block_table;  /* [num_seqs][max_blocks_per_seq]; entries past ceil(L_s/page_size)
+                                    are never read */
+    const int32_t* seq_lens;     /* [num_seqs] L_s */
+    const int32_t* cu_q_lens;    /* [num_seqs+1] prefix sums of n_s; prefill only (decode: NULL) */
+    const int32_t* spans;        /* [num_seqs][S][2] half-open absolute key ranges [a,b); clipped to the
+                                    visible keys; a >= b is an empty span.  NULL = no probe */
+    const float*   steer_vec;    /* fp32 [Hq][D]; NULL = no steering */
+    void*          out;          /* bf16 [total_q][Hq][D] */
+    float*         span_mass;    /* fp32 [rows][P][S]; rows = total_q (ALL) or num_seqs (LAST, decode);
+                                    P = number of nonzero head_mask entries; the slot of a probed head is
+                                    its rank among the probed heads in ascending head order */
+    void*          workspace;    /* scratch of at least hook_attn_workspace_bytes(); 256-byte aligned */
+    size_t         workspace_bytes;
+    int32_t*       status;       /* optional: one int32, set to a negative HOOK_ATTN_ERR_* code by the
+                                    device on a detected fault; the caller zeroes it beforehand */
+
+    /* ---- HOST arrays, read during the call and copied into the kernel parameters ---- */
+    const uint8_t* head_mask;    /* host [Hq]; nonzero = probed head.  NULL = no probe */
+    const float*   alpha;        /* host [Hq]; 0 = head not steered.  NULL = no steering */
+} hook_attn_params;
+
+/* Create / destroy the per-device handle.  `device` is a CUDA device ordinal.  Creation queries
+ * device properties and configures the kernels; it fails with HOOK_ATTN_ERR_UNSUPPORTED on a
+ * device that is not compute capability 10.x, HOOK_ATTN_ERR_CUDA if no device is usable. */
+int hook_attn_create(hook_attn_handle** handle, int device);
+int hook_attn_destroy(hook_attn_handle* handle);
+
+/* Bytes of scratch the call described by `p` needs (only the shape fields are read).
+ * is_decode != 0 sizes hook_attn_decode, 0 sizes hook_attn_prefill.  Returns 0 when the call needs
+ * no scratch or when the shapes are invalid. */
+size_t hook_attn_workspace_bytes(const hook_attn_params* p, int is_decode);
+
+/* Prefill / chunked prefill: n_s >= 0 rows per sequence given by cu_q_lens, n_s <= L_s.
+ * (Section 2.2 recompute + Section 2 steering, fused into the attention forward.) */
+int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
+
+/* Decode: exactly one query row per sequence (total_q == num_seqs, cu_q_lens ignored); keys are
+ * split into chunks that are reduced independently and merged in a fixed order, so results are
+ * bit-identical from run to run.  span_mass has one row per sequence. */
+int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
+
+/* Human-readable name of a return / status code. */
+const char* hook_attn_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HOOK_ATTN_H_ */

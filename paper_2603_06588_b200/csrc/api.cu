@@ -1,0 +1,194 @@
+// C ABI of the hooked paged-attention library: argument validation, workspace sizing, dispatch.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace hook_attn {
+// decode.cu
+cudaError_t configure_decode();
+cudaError_t launch_decode(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st);
+size_t decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim, int max_chunks);
+int decode_pick_chunk(int num_seqs, int Hkv, int max_blocks, int num_sms);
+// prefill_mma.cu
+cudaError_t configure_prefill_mma();
+cudaError_t launch_prefill_mma(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st);
+int prefill_mma_tiles_upper_bound(int total_q, int num_seqs);
+}  // namespace hook_attn
+
+using namespace hook_attn;
+
+struct hook_attn_handle {
+    int device;
+    int num_sms;
+    int cc_major, cc_minor;
+};
+
+namespace {
+
+constexpr int kDefaultSMs = 148;
+
+int validate_common(const hook_attn_params* p, bool decode)
+{
+    if (!p) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (p->num_seqs < 0 || p->total_q < 0 || p->num_q_heads <= 0 || p->num_kv_heads <= 0 || p->head_dim <= 0 ||
+        p->page_size <= 0 || p->num_blocks < 0 || p->max_blocks_per_seq < 0 || p->num_spans < 0)
+        return HOOK_ATTN_ERR_INVALID_ARG;
+    if (p->num_q_heads % p->num_kv_heads != 0) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (decode && p->total_q != p->num_seqs) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (p->probe_rows != HOOK_PROBE_ROWS_ALL && p->probe_rows != HOOK_PROBE_ROWS_LAST) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (p->head_dim != 64 && p->head_dim != 128) return HOOK_ATTN_ERR_UNSUPPORTED;
+    if (p->page_size != kPage) return HOOK_ATTN_ERR_UNSUPPORTED;
+    if (p->num_q_heads > kMaxHeads) return HOOK_ATTN_ERR_UNSUPPORTED;
+    if (p->num_q_heads / p->num_kv_heads > kMaxGroup) return HOOK_ATTN_ERR_UNSUPPORTED;
+    if (p->num_spans > kMaxSpans) return HOOK_ATTN_ERR_UNSUPPORTED;
+    if (p->num_seqs > 65535) return HOOK_ATTN_ERR_UNSUPPORTED;
+    return HOOK_ATTN_OK;
+}
+
+bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+
+// Fills the kernel arguments; returns a HOOK_ATTN_* code.
+int prepare(const hook_attn_params* p, bool decode, KernelArgs& a, HeadCfg& hc)
+{
+    int rc = validate_common(p, decode);
+    if (rc != HOOK_ATTN_OK) return rc;
+    if (p->num_seqs == 0 || p->total_q == 0) return HOOK_ATTN_OK;   // nothing to do (caller checks total_q)
+    if (!p->q || !p->k_cache || !p->v_cache || !p->block_table || !p->seq_lens || !p->out) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (!decode && !p->cu_q_lens) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (p->kv_block_stride <= 0 || p->kv_token_stride <= 0 || p->kv_head_stride <= 0) return HOOK_ATTN_ERR_INVALID_ARG;
+    if ((p->kv_block_stride | p->kv_token_stride | p->kv_head_stride) & 7) return HOOK_ATTN_ERR_UNSUPPORTED;
+    if (!aligned16(p->q) || !aligned16(p->k_cache) || !aligned16(p->v_cache) || !aligned16(p->out)) return HOOK_ATTN_ERR_UNSUPPORTED;
+
+    memset(&hc, 0, sizeof hc);
+    int probed = 0;
+    bool any_steer = false;
+    for (int h = 0; h < kMaxHeads; ++h) hc.slot[h] = -1;
+    for (int h = 0; h < p->num_q_heads; ++h) {
+        if (p->head_mask && p->head_mask[h]) hc.slot[h] = (int8_t)probed++;
+        if (p->alpha && p->alpha[h] != 0.0f) {
+            if (!isfinite(p->alpha[h])) return HOOK_ATTN_ERR_INVALID_ARG;
+            hc.alpha[h] = p->alpha[h];
+            any_steer = true;
+        }
+    }
+    const bool any_probe = probed > 0 && p->num_spans > 0;
+    if (any_probe && (!p->spans || !p->span_mass)) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (any_steer && !p->steer_vec) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (!any_probe) for (int h = 0; h < kMaxHeads; ++h) hc.slot[h] = -1;
+
+    memset(&a, 0, sizeof a);
+    a.q = static_cast<const __nv_bfloat16*>(p->q);
+    a.k = static_cast<const __nv_bfloat16*>(p->k_cache);
+    a.v = static_cast<const __nv_bfloat16*>(p->v_cache);
+    a.bs = p->kv_block_stride; a.ts = p->kv_token_stride; a.hs = p->kv_head_stride;
+    a.block_table = p->block_table; a.seq_lens = p->seq_lens; a.cu_q_lens = p->cu_q_lens;
+    a.spans = p->spans; a.steer = p->steer_vec;
+    a.out = static_cast<__nv_bfloat16*>(p->out);
+    a.mass = p->span_mass;
+    a.ws = static_cast<float*>(p->workspace);
+    a.status = p->status;
+    a.num_seqs = p->num_seqs; a.total_q = p->total_q; a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads;
+    a.G = p->num_q_heads / p->num_kv_heads;
+    a.num_blocks = p->num_blocks; a.max_blocks = p->max_blocks_per_seq;
+    a.S = any_probe ? p->num_spans : 0; a.P = probed; a.probe_rows = p->probe_rows;
+    const float scale = (p->scale > 0.f) ? p->scale : 1.0f / sqrtf((float)p->head_dim);
+    a.scale_log2 = scale * 1.4426950408889634f;
+    a.any_probe = any_probe; a.any_steer = any_steer;
+    return HOOK_ATTN_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int hook_attn_create(hook_attn_handle** handle, int device)
+{
+    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    *handle = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        (void)cudaGetLastError();
+        return HOOK_ATTN_ERR_CUDA;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return HOOK_ATTN_ERR_CUDA;
+    if (prop.major != 10) return HOOK_ATTN_ERR_UNSUPPORTED;
+    int prev = 0;
+    cudaGetDevice(&prev);
+    if (cudaSetDevice(device) != cudaSuccess) return HOOK_ATTN_ERR_CUDA;
+    cudaError_t e = configure_decode();
+    if (e == cudaSuccess) e = configure_prefill_mma();
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) return HOOK_ATTN_ERR_CUDA;
+    hook_attn_handle* h = new hook_attn_handle;
+    h->device = device;
+    h->num_sms = prop.multiProcessorCount;
+    h->cc_major = prop.major;
+    h->cc_minor = prop.minor;
+    *handle = h;
+    return HOOK_ATTN_OK;
+}
+
+int hook_attn_destroy(hook_attn_handle* handle)
+{
+    delete handle;
+    return HOOK_ATTN_OK;
+}
+
+size_t hook_attn_workspace_bytes(const hook_attn_params* p, int is_decode)
+{
+    if (validate_common(p, is_decode != 0) != HOOK_ATTN_OK) return 0;
+    if (!is_decode) return 0;
+    const int G = p->num_q_heads / p->num_kv_heads;
+    const int chunk = decode_pick_chunk(p->num_seqs, p->num_kv_heads, p->max_blocks_per_seq, kDefaultSMs);
+    const int max_chunks = (p->max_blocks_per_seq * kPage + chunk - 1) / chunk;
+    return decode_workspace_bytes(p->num_seqs, p->num_kv_heads, G, p->head_dim, max_chunks > 0 ? max_chunks : 1);
+}
+
+int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream)
+{
+    KernelArgs a;
+    HeadCfg hc;
+    int rc = prepare(p, false, a, hc);     // argument errors are reported before anything else
+    if (rc != HOOK_ATTN_OK) return rc;
+    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (p->num_seqs == 0 || p->total_q == 0) return HOOK_ATTN_OK;
+    a.total_tiles = prefill_mma_tiles_upper_bound(p->total_q, p->num_seqs);
+    cudaError_t e = launch_prefill_mma(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
+}
+
+int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream)
+{
+    KernelArgs a;
+    HeadCfg hc;
+    int rc = prepare(p, true, a, hc);
+    if (rc != HOOK_ATTN_OK) return rc;
+    if (p->num_seqs > 0 && p->max_blocks_per_seq == 0) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (p->num_seqs == 0) return handle ? HOOK_ATTN_OK : HOOK_ATTN_ERR_INVALID_ARG;
+    a.chunk = decode_pick_chunk(p->num_seqs, p->num_kv_heads, p->max_blocks_per_seq, kDefaultSMs);
+    a.max_chunks = (p->max_blocks_per_seq * kPage + a.chunk - 1) / a.chunk;
+    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, a.max_chunks);
+    if (!p->workspace || p->workspace_bytes < need) return HOOK_ATTN_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(p->workspace) & 15u) return HOOK_ATTN_ERR_WORKSPACE;
+    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    cudaError_t e = launch_decode(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
+}
+
+const char* hook_attn_strerror(int code)
+{
+    switch (code) {
+        case HOOK_ATTN_OK: return "ok";
+        case HOOK_ATTN_ERR_INVALID_ARG: return "invalid argument";
+        case HOOK_ATTN_ERR_UNSUPPORTED: return "unsupported shape, layout or device";
+        case HOOK_ATTN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case HOOK_ATTN_ERR_CUDA: return "CUDA call failed";
+        case HOOK_ATTN_ERR_TIMEOUT: return "bounded wait ran out on the device";
+        case HOOK_ATTN_ERR_BOUNDS: return "block id or sequence length out of range";
+        default: return "unknown code";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,357 @@
+// Split-K decode of the hooked paged attention: one query row per sequence.
+//
+// Kernel 1 (decode_splitk): one CTA per (key chunk, KV head, sequence).  The G <= 8 query heads
+// that share the KV head are processed together with warp-level tensor-core tiles in the
+// transposed orientation: a 16-key page is the M dimension, the query heads are the N = 8
+// dimension (S^T = K Q^T, O^T = V^T P^T), so no padding work is spent on the single query row.
+// Each warp streams its own pages through a private multi-stage cp.async pipeline (16-byte
+// copies, zero-filled past the end of the sequence), keeps an online softmax per head, and
+// carries the span masses of the probe as extra accumulators in the same frame as the running
+// sum.  The four warps are merged in shared memory and the chunk's partial (m, l, o[D], s[S]) is
+// written to the workspace.
+//
+// Kernel 2 (decode_merge): one CTA per (query head, sequence) merges the chunk partials in chunk
+// order (run-to-run bit-identical), normalises, applies the steering add and stores.
+#include "common.cuh"
+
+namespace hook_attn {
+
+constexpr int kDecWarps = 4;
+constexpr int kDecStages = 3;
+constexpr int kPartPad = 16;   // floats after o[D] in a partial: m, l, s[0..7], padding
+
+template <int HD>
+constexpr int decode_smem_bytes()
+{
+    return kDecWarps * kDecStages * 2 * kPage * HD * 2;
+}
+
+__host__ __device__ inline size_t decode_partial_stride(int head_dim) { return (size_t)head_dim + kPartPad; }
+
+template <int HD, int NS>
+__global__ void __launch_bounds__(kDecWarps * 32) decode_splitk_kernel(const KernelArgs a, const HeadCfg hc)
+{
+    constexpr int ROWB = HD * 2;            // bytes per K/V row
+    constexpr int TILEB = kPage * ROWB;     // bytes per 16-key tile
+    constexpr int CPR = HD / 8;             // 16-byte chunks per row
+    constexpr int RPI = 32 / CPR;           // rows covered by one warp-wide copy instruction
+    constexpr int KS = HD / 16;             // k-steps of the score product / d-blocks of the output
+    constexpr int OSTR = HD + 4;            // padded row of the cross-warp reduction buffer
+
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ int sh_span[2 * kMaxSpans];
+    __shared__ float sh_m[kDecWarps][8];
+    __shared__ float sh_small[kDecWarps][8][2 + kMaxSpans];
+
+    const int s = blockIdx.z, kvh = blockIdx.y, c = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+    const int G = a.G;
+
+    const int L = a.seq_lens[s];
+    if (L <= 0 || L > a.max_blocks * kPage) return;   // reported and zero-filled by the merge kernel
+    const int start = c * a.chunk;
+    if (start >= L) return;
+    const int end = min(L, start + a.chunk);
+    const int ntiles = (end - start + kPage - 1) / kPage;
+
+    bool probe = false;
+    if constexpr (NS > 0) {
+        for (int i = 0; i < G; ++i) probe |= (hc.slot[kvh * G + i] >= 0);
+        if ((int)threadIdx.x < 2 * NS) {
+            const int j = threadIdx.x >> 1;
+            sh_span[threadIdx.x] = (probe && j < a.S) ? a.spans[((int64_t)s * a.S + j) * 2 + (threadIdx.x & 1)] : 0;
+        }
+    }
+    __syncthreads();
+
+    // B fragments of Q^T (k = d, n = head): head g of the group, zero for padding heads.
+    uint32_t qb[KS][2];
+    {
+        const __nv_bfloat16* qrow = a.q + ((int64_t)s * a.Hq + kvh * G + g) * HD;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            qb[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * tq) : 0u;
+            qb[ks][1] = (g < G) ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * tq) : 0u;
+        }
+    }
+
+    const uint32_t wbase = smem_u32(smem) + warp * (kDecStages * 2 * TILEB);
+    const int32_t* bt = a.block_table + (int64_t)s * a.max_blocks;
+    const int my_tiles = (ntiles > warp) ? (ntiles - warp + kDecWarps - 1) / kDecWarps : 0;
+
+    auto issue = [&](int it) {
+        if (it < my_tiles) {
+            const int key0 = start + (warp + it * kDecWarps) * kPage;
+            int page = bt[key0 / kPage];
+            bool page_ok = (page >= 0 && page < a.num_blocks);
+            if (!page_ok) { report(a.status, HOOK_ATTN_ERR_BOUNDS); page = 0; }
+            const uint32_t kdst = wbase + (it % kDecStages) * (2 * TILEB);
+            const uint32_t vdst = kdst + TILEB;
+            const int64_t base = (int64_t)page * a.bs + (int64_t)kvh * a.hs;
+#pragma unroll
+            for (int i = 0; i < kPage / RPI; ++i) {
+                const int r = i * RPI + lane / CPR;
+                const int cc = lane % CPR;
+                const bool ok = page_ok && (key0 + r < L);
+                const int64_t off = base + (int64_t)r * a.ts + cc * 8;
+                cp_async16(kdst + swz<ROWB>(r, cc), a.k + off, ok);
+                cp_async16(vdst + swz<ROWB>(r, cc), a.v + off, ok);
+            }
+        }
+        cp_async_commit();
+    };
+
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float o[KS][4];
+#pragma unroll
+    for (int i = 0; i < KS; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float sm[NS > 0 ? NS : 1][2];
+#pragma unroll
+    for (int j = 0; j < (NS > 0 ? NS : 1); ++j) sm[j][0] = sm[j][1] = 0.f;
+
+#pragma unroll
+    for (int i = 0; i < kDecStages - 1; ++i) issue(i);
+
+    for (int it = 0; it < my_tiles; ++it) {
+        issue(it + kDecStages - 1);
+        cp_async_wait<kDecStages - 1>();
+        __syncwarp();
+
+        const int key0 = start + (warp + it * kDecWarps) * kPage;
+        const uint32_t kt = wbase + (it % kDecStages) * (2 * TILEB);
+        const uint32_t vt = kt + TILEB;
+
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            uint32_t af[4];
+            ldmatrix_x4(af, kt + swz<ROWB>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)));
+            mma_bf16_16816(sc, af, qb[ks][0], qb[ks][1]);
+        }
+        const int t0 = key0 + g, t1 = t0 + 8;
+        const float x0 = (t0 < L) ? sc[0] * a.scale_log2 : -INFINITY;   // (key t0, head 2tq)
+        const float x1 = (t0 < L) ? sc[1] * a.scale_log2 : -INFINITY;   // (key t0, head 2tq+1)
+        const float x2 = (t1 < L) ? sc[2] * a.scale_log2 : -INFINITY;   // (key t1, head 2tq)
+        const float x3 = (t1 < L) ? sc[3] * a.scale_log2 : -INFINITY;   // (key t1, head 2tq+1)
+        float mx0 = fmaxf(x0, x2), mx1 = fmaxf(x1, x3);
+#pragma unroll
+        for (int d = 4; d <= 16; d <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, d));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, d));
+        }
+        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: key0 < L
+        const float c0 = fast_exp2(m0 - mn0), c1 = fast_exp2(m1 - mn1);
+        m0 = mn0; m1 = mn1;
+        const float p0 = fast_exp2(x0 - mn0), p1 = fast_exp2(x1 - mn1);
+        const float p2 = fast_exp2(x2 - mn0), p3 = fast_exp2(x3 - mn1);
+        l0 = l0 * c0 + (p0 + p2);
+        l1 = l1 * c1 + (p1 + p3);
+#pragma unroll
+        for (int i = 0; i < KS; ++i) { o[i][0] *= c0; o[i][1] *= c1; o[i][2] *= c0; o[i][3] *= c1; }
+
+        if (NS > 0 && probe) {
+#pragma unroll
+            for (int j = 0; j < NS; ++j) {
+                const int sa = sh_span[2 * j], sb = sh_span[2 * j + 1];
+                float add0 = 0.f, add1 = 0.f;
+                if (sb > key0 && sa < key0 + kPage) {
+                    const bool in0 = (t0 >= sa) && (t0 < sb), in1 = (t1 >= sa) && (t1 < sb);
+                    add0 = (in0 ? p0 : 0.f) + (in1 ? p2 : 0.f);
+                    add1 = (in0 ? p1 : 0.f) + (in1 ? p3 : 0.f);
+                }
+                sm[j][0] = sm[j][0] * c0 + add0;
+                sm[j][1] = sm[j][1] * c1 + add1;
+            }
+        }
+
+        // P^T as the B operand (k = key, n = head): transpose the two 8x8 blocks across lanes.
+        const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
+        const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
+#pragma unroll
+        for (int i = 0; i < KS; ++i) {
+            uint32_t af[4];
+            ldmatrix_x4_trans(af, vt + swz<ROWB>((lane & 7) + (lane >> 4) * 8, 2 * i + ((lane >> 3) & 1)));
+            mma_bf16_16816(o[i], af, pb0, pb1);
+        }
+        __syncwarp();
+    }
+    cp_async_wait<0>();
+
+    // per-thread partial sums -> per-warp sums (lanes with the same tq hold the same heads)
+#pragma unroll
+    for (int d = 4; d <= 16; d <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, d);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, d);
+        if (NS > 0) {
+#pragma unroll
+            for (int j = 0; j < NS; ++j) {
+                sm[j][0] += __shfl_xor_sync(0xffffffffu, sm[j][0], d);
+                sm[j][1] += __shfl_xor_sync(0xffffffffu, sm[j][1], d);
+            }
+        }
+    }
+
+    // ---- merge the four warps ----
+    if (g == 0) { sh_m[warp][2 * tq] = m0; sh_m[warp][2 * tq + 1] = m1; }
+    __syncthreads();   // also: every warp has drained its pipeline, the stage buffers are free
+    float M0 = sh_m[0][2 * tq], M1 = sh_m[0][2 * tq + 1];
+#pragma unroll
+    for (int w = 1; w < kDecWarps; ++w) { M0 = fmaxf(M0, sh_m[w][2 * tq]); M1 = fmaxf(M1, sh_m[w][2 * tq + 1]); }
+    const float f0 = fast_exp2(m0 - M0), f1 = fast_exp2(m1 - M1);   // warp without tiles: m = -inf -> 0
+
+    float* red = reinterpret_cast<float*>(smem);   // [warps][8 heads][OSTR]
+#pragma unroll
+    for (int i = 0; i < KS; ++i) {
+        float* r0 = red + (warp * 8 + 2 * tq) * OSTR;
+        r0[16 * i + g] = o[i][0] * f0;
+        r0[OSTR + 16 * i + g] = o[i][1] * f1;
+        r0[16 * i + 8 + g] = o[i][2] * f0;
+        r0[OSTR + 16 * i + 8 + g] = o[i][3] * f1;
+    }
+    if (g == 0) {
+        sh_small[warp][2 * tq][0] = M0;
+        sh_small[warp][2 * tq + 1][0] = M1;
+        sh_small[warp][2 * tq][1] = l0 * f0;
+        sh_small[warp][2 * tq + 1][1] = l1 * f1;
+        if (NS > 0) {
+#pragma unroll
+            for (int j = 0; j < NS; ++j) {
+                sh_small[warp][2 * tq][2 + j] = sm[j][0] * f0;
+                sh_small[warp][2 * tq + 1][2 + j] = sm[j][1] * f1;
+            }
+        }
+    }
+    __syncthreads();
+
+    const size_t pstride = decode_partial_stride(HD);
+    float* part = a.ws + (((size_t)s * a.Hkv + kvh) * a.max_chunks + c) * G * pstride;
+    for (int idx = threadIdx.x; idx < G * HD; idx += kDecWarps * 32) {
+        const int h = idx / HD, d = idx % HD;
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kDecWarps; ++w) acc += red[(w * 8 + h) * OSTR + d];
+        part[h * pstride + d] = acc;
+    }
+    for (int idx = threadIdx.x; idx < G * (2 + NS); idx += kDecWarps * 32) {
+        const int h = idx / (2 + NS), e = idx % (2 + NS);
+        float val;
+        if (e == 0) {
+            val = sh_small[0][h][0];
+        } else {
+            val = 0.f;
+#pragma unroll
+            for (int w = 0; w < kDecWarps; ++w) val += sh_small[w][h][e];
+        }
+        part[h * pstride + HD + e] = val;
+    }
+}
+
+template <int HD>
+__global__ void __launch_bounds__(128) decode_merge_kernel(const KernelArgs a, const HeadCfg hc)
+{
+    const int h = blockIdx.x, s = blockIdx.y;
+    const int G = a.G, kvh = h / G, gi = h % G;
+    const int L = a.seq_lens[s];
+    const int d = threadIdx.x;
+    __nv_bfloat16* orow = a.out + ((int64_t)s * a.Hq + h) * HD;
+    const int slot = hc.slot[h];
+    float* mrow = (slot >= 0 && a.S > 0) ? a.mass + ((int64_t)s * a.P + slot) * a.S : nullptr;
+
+    if (L <= 0 || L > a.max_blocks * kPage) {
+        if (threadIdx.x == 0) report(a.status, L <= 0 ? HOOK_ATTN_ERR_INVALID_ARG : HOOK_ATTN_ERR_BOUNDS);
+        if (d < HD) orow[d] = __float2bfloat16(0.f);
+        if (mrow && d < a.S) mrow[d] = 0.f;
+        return;
+    }
+    const int nchunks = (L + a.chunk - 1) / a.chunk;
+    const size_t pstride = decode_partial_stride(HD);
+    const float* part = a.ws + ((((size_t)s * a.Hkv + kvh) * a.max_chunks) * G + gi) * pstride;
+    const size_t cstride = (size_t)G * pstride;
+
+    float M = -INFINITY;
+    for (int c = 0; c < nchunks; ++c) M = fmaxf(M, part[c * cstride + HD]);
+    float acc = 0.f, lsum = 0.f, macc = 0.f;
+    for (int c = 0; c < nchunks; ++c) {
+        const float* pc = part + c * cstride;
+        const float w = fast_exp2(pc[HD] - M);
+        lsum += w * pc[HD + 1];
+        if (d < HD) acc += w * pc[d];
+        if (mrow && d < a.S) macc += w * pc[HD + 2 + d];
+    }
+    const float inv = 1.f / lsum;
+    if (d < HD) {
+        float val = acc * inv;
+        const float al = hc.alpha[h];
+        if (al != 0.f) val += al * a.steer[(int64_t)h * HD + d];
+        orow[d] = __float2bfloat16(val);
+    }
+    if (mrow && d < a.S) mrow[d] = macc * inv;
+}
+
+// ------------------------------------------------------------------------------------------
+template <int HD, int NS>
+static cudaError_t launch_decode_t(const KernelArgs& a, const HeadCfg& hc, cudaStream_t st)
+{
+    dim3 grid(a.max_chunks, a.Hkv, a.num_seqs);
+    decode_splitk_kernel<HD, NS><<<grid, kDecWarps * 32, decode_smem_bytes<HD>(), st>>>(a, hc);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    decode_merge_kernel<HD><<<dim3(a.Hq, a.num_seqs), 128, 0, st>>>(a, hc);
+    return cudaGetLastError();
+}
+
+template <int HD, int NS>
+static cudaError_t configure_one()
+{
+    return cudaFuncSetAttribute(decode_splitk_kernel<HD, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                decode_smem_bytes<HD>());
+}
+
+// Opt in to the dynamic shared memory the split-K kernels use (per device; called with the
+// device current when a handle is created).
+cudaError_t configure_decode()
+{
+    cudaError_t e;
+#define HOOK_CFG(HD, NS) if ((e = configure_one<HD, NS>()) != cudaSuccess) return e;
+    HOOK_CFG(64, 0) HOOK_CFG(64, 2) HOOK_CFG(64, 4) HOOK_CFG(64, 8)
+    HOOK_CFG(128, 0) HOOK_CFG(128, 2) HOOK_CFG(128, 4) HOOK_CFG(128, 8)
+#undef HOOK_CFG
+    return cudaSuccess;
+}
+
+// Keys per split-K chunk, from host-known bounds only (sequence lengths live on the device):
+// the largest power-of-two chunk that still leaves at least eight CTAs per SM in the grid.
+int decode_pick_chunk(int num_seqs, int Hkv, int max_blocks, int num_sms)
+{
+    const long max_keys = (long)max_blocks * kPage;
+    int chunk = 2048;
+    while (chunk > 256) {
+        const long ctas = (long)num_seqs * Hkv * ((max_keys + chunk - 1) / chunk);
+        if (ctas >= 8L * num_sms) break;
+        chunk >>= 1;
+    }
+    return chunk;
+}
+
+size_t decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim, int max_chunks)
+{
+    return (size_t)num_seqs * Hkv * max_chunks * G * decode_partial_stride(head_dim) * sizeof(float);
+}
+
+cudaError_t launch_decode(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st)
+{
+    const int ns = !a.any_probe ? 0 : (a.S <= 2 ? 2 : (a.S <= 4 ? 4 : 8));
+#define HOOK_DISPATCH(HD)                                                         \
+    switch (ns) {                                                                 \
+        case 0: return launch_decode_t<HD, 0>(a, hc, st);                         \
+        case 2: return launch_decode_t<HD, 2>(a, hc, st);                         \
+        case 4: return launch_decode_t<HD, 4>(a, hc, st);                         \
+        default: return launch_decode_t<HD, 8>(a, hc, st);                        \
+    }
+    if (head_dim == 128) { HOOK_DISPATCH(128) }
+    HOOK_DISPATCH(64)
+#undef HOOK_DISPATCH
+}
+
+}  // namespace hook_attn

@@ -1,0 +1,289 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle, element by element
+on the same seeded inputs.
+
+Tolerances (stated by the target): max |out_bf16 - oracle| <= 2e-2, max |span_mass - oracle| <= 1e-3.
+Index handling (block tables, page slots, span edges, compact probe slots) is checked bit-exactly
+through cases whose result is a single value row or an exact 0/1 mass.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle
+from paper_2603_06588_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_OUT = 2e-2
+TOL_MASS = 1e-3
+
+
+@pytest.fixture(scope="module")
+def eng():
+    return binding.HookAttn(0)
+
+
+def run_gpu(eng, case, **over):
+    kw = binding.case_to_device(case)
+    kw.update(over)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fn = eng.hook_attn_decode if case.is_decode else eng.hook_attn_prefill
+    out, mass = fn(status=status, **kw)
+    torch.cuda.synchronize()
+    return out, mass, int(status.item())
+
+
+def mass_rows(case, rows):
+    """Map evaluated query rows to rows of the GPU span_mass tensor (None = not stored)."""
+    if case.is_decode or case.probe_rows == inputs.PROBE_ROWS_LAST:
+        cu = case.cu_q_lens.tolist()
+        last = {cu[s + 1] - 1: s for s in range(case.num_seqs) if cu[s + 1] > cu[s]}
+        return [last.get(r) for r in rows]
+    return list(rows)
+
+
+def check(eng, case, rows=None, tol_out=TOL_OUT, tol_mass=TOL_MASS):
+    out, mass, status = run_gpu(eng, case)
+    assert status == 0, binding.strerror(status)
+    ref_out, ref_mass = oracle.run(case, rows)
+    idx = list(range(case.total_q)) if rows is None else list(rows)
+    got = out.float().cpu().numpy().astype(np.float64)[idx]
+    assert np.isfinite(got).all()
+    err_o = np.abs(got - ref_out).max() if got.size else 0.0
+    assert err_o <= tol_out, f"{case.name}: out error {err_o}"
+    err_m = 0.0
+    if ref_mass is not None:
+        gm = mass.cpu().numpy().astype(np.float64)
+        mr = mass_rows(case, idx)
+        sel = [i for i, r in enumerate(mr) if r is not None]
+        assert sel, "no probed row among the checked rows"
+        g = gm[[mr[i] for i in sel]]
+        assert np.isfinite(g).all()
+        err_m = np.abs(g - ref_mass[sel]).max()
+        assert err_m <= tol_mass, f"{case.name}: span_mass error {err_m}"
+    return err_o, err_m
+
+
+# ------------------------------------------------------------------ the five named workloads
+def test_config1_tiny_prefill(eng):
+    check(eng, inputs.config1_tiny_prefill(poison=True))
+
+
+def test_config2_decode_full(eng):
+    check(eng, inputs.config2_decode(poison=True))
+
+
+def test_config3_prefill_midsize_all_rows(eng):
+    check(eng, inputs.config3_prefill(layer=0, num_seqs=2, tokens=1024, poison=True, force_probe=True))
+
+
+@pytest.mark.parametrize("layer", [0, 5])
+def test_config3_prefill_full_size_sampled_rows(eng, layer):
+    case = inputs.config3_prefill(layer=layer, force_probe=True)
+    check(eng, case, rows=inputs.sample_rows(case, extra_random=8))
+
+
+def test_config4_mixed_decode_full_size(eng):
+    case = inputs.config4_decode()
+    assert float(case.alpha.abs().max()) <= 2.0
+    err_o, _ = check(eng, case)
+    ref_out, _ = oracle.run(case)
+    assert np.abs(ref_out).max() < 8.0      # bf16 spacing stays below the output tolerance
+
+
+def test_config4_mixed_prefill_chunks_sampled_rows(eng):
+    case = inputs.config4_prefill()
+    check(eng, case, rows=inputs.sample_rows(case, extra_random=16))
+
+
+def test_config4_mixed_prefill_small_all_rows(eng):
+    check(eng, inputs.config4_prefill(chunks=2, n=200, ctx=333, poison=True))
+
+
+def test_config5_long_prefill_small_all_rows(eng):
+    check(eng, inputs.config5_prefill(num_seqs=2, tokens=640, poison=True))
+
+
+def test_config5_long_prefill_full_size_sampled_rows(eng):
+    case = inputs.config5_prefill()
+    check(eng, case, rows=inputs.sample_rows(case, extra_random=4))
+
+
+@pytest.mark.parametrize("step", [0, 127])
+def test_config5_long_decode_full_size(eng, step):
+    check(eng, inputs.config5_decode(step=step))
+
+
+# ------------------------------------------------------------------------------- edge cases
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 8, 64), (8, 1, 64), (14, 2, 128), (6, 2, 128), (32, 8, 128), (64, 8, 128)])
+def test_decode_shapes_and_ragged_lengths(eng, Hq, Hkv, D):
+    lens = [1, 2, 15, 16, 17, 31, 33, 63, 64, 65, 255, 256, 257, 1023, 1025, 3000]
+    g = inputs._gen(Hq * 131 + D)
+    alpha = torch.zeros(Hq)
+    alpha[::3] = 0.7
+    case = inputs.make_case("dec_edge", is_decode=True, seq_lens=lens, q_lens=[1] * len(lens),
+                            num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, seed=77 + Hq, num_spans=3,
+                            head_mask=inputs.choose_heads(Hq, max(1, Hq // 2), g), alpha=alpha, steer=True,
+                            probe_rows=inputs.PROBE_ROWS_LAST, poison=True)
+    check(eng, case)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 8, 64), (4, 1, 64), (14, 2, 128), (8, 2, 128)])
+def test_prefill_shapes_ragged_and_chunked(eng, Hq, Hkv, D):
+    seq_lens = [1, 17, 64, 65, 130, 300, 77, 200]
+    q_lens = [1, 17, 64, 65, 130, 100, 0, 3]            # full, chunked, empty, short tail
+    g = inputs._gen(Hq * 17 + D)
+    alpha = torch.zeros(Hq)
+    alpha[1::2] = -1.25
+    case = inputs.make_case("pf_edge", is_decode=False, seq_lens=seq_lens, q_lens=q_lens,
+                            num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, seed=91 + Hq, num_spans=4,
+                            head_mask=inputs.choose_heads(Hq, max(1, Hq // 2), g), alpha=alpha, steer=True,
+                            probe_rows=inputs.PROBE_ROWS_ALL, poison=True)
+    check(eng, case)
+
+
+def test_prefill_last_token_mode_equals_last_row_of_all_tokens(eng):
+    case = inputs.make_case("pf_last", is_decode=False, seq_lens=[150, 64, 9], q_lens=[150, 20, 9],
+                            num_q_heads=8, num_kv_heads=2, head_dim=128, seed=5, num_spans=3,
+                            head_mask=torch.tensor([1, 0, 1, 1, 0, 0, 0, 1], dtype=torch.uint8), poison=True)
+    out_a, mass_a, st = run_gpu(eng, case)
+    assert st == 0
+    last = inputs.replace(case, probe_rows=inputs.PROBE_ROWS_LAST)
+    out_l, mass_l, st = run_gpu(eng, last)
+    assert st == 0 and mass_l.shape == (3, 4, 3)
+    assert torch.equal(out_a, out_l)
+    assert torch.equal(mass_l, mass_a[[r for r in oracle.last_rows(case)]])
+    check(eng, last)
+
+
+def test_probes_do_not_change_the_output_bits_and_runs_are_deterministic(eng):
+    for case in (inputs.config2_decode(num_seqs=16, lo=100, hi=2500),
+                 inputs.config3_prefill(layer=2, num_seqs=2, tokens=300, force_probe=True)):
+        steer_only = inputs.replace(case, spans=None, head_mask=None, num_spans=0)
+        out_h, mass_h, _ = run_gpu(eng, case)
+        out_p, _, _ = run_gpu(eng, steer_only)
+        out_h2, mass_h2, _ = run_gpu(eng, case)
+        assert torch.equal(out_h.view(torch.int16), out_p.view(torch.int16))
+        assert torch.equal(out_h.view(torch.int16), out_h2.view(torch.int16))
+        assert torch.equal(mass_h, mass_h2)
+
+
+def test_hooks_disabled_is_plain_attention(eng):
+    case = inputs.config2_decode(num_seqs=8, lo=50, hi=900)
+    zero = inputs.replace(case, alpha=torch.zeros(case.num_q_heads), head_mask=torch.zeros(case.num_q_heads, dtype=torch.uint8))
+    out_z, mass_z, st = run_gpu(eng, zero)
+    out_n, mass_n, _ = run_gpu(eng, case.without_hooks())
+    assert st == 0 and mass_z is None and mass_n is None
+    assert torch.equal(out_z.view(torch.int16), out_n.view(torch.int16))
+    check(eng, case.without_hooks())
+
+
+def test_page_permutation_is_bitwise_invariant(eng):
+    for case in (inputs.config2_decode(num_seqs=8, lo=30, hi=1200),
+                 inputs.make_case("pf_perm", is_decode=False, seq_lens=[200, 90], q_lens=[200, 30], num_q_heads=8,
+                                  num_kv_heads=2, head_dim=128, seed=8, num_spans=2,
+                                  head_mask=torch.ones(8, dtype=torch.uint8))):
+        out, mass, _ = run_gpu(eng, case)
+        g = inputs._gen(5)
+        perm = torch.randperm(case.num_blocks, generator=g)
+        inv = torch.empty_like(perm)
+        inv[perm] = torch.arange(case.num_blocks)
+        bt = case.block_table.clone()
+        valid = bt >= 0
+        bt[valid] = inv[bt[valid].long()].to(torch.int32)
+        moved = inputs.replace(case, k_cache=case.k_cache[perm].contiguous(),
+                               v_cache=case.v_cache[perm].contiguous(), block_table=bt)
+        out_p, mass_p, _ = run_gpu(eng, moved)
+        assert torch.equal(out.view(torch.int16), out_p.view(torch.int16)) and torch.equal(mass, mass_p)
+
+
+@pytest.mark.parametrize("decode", [True, False])
+def test_dominating_key_returns_its_value_row_bit_exactly(eng, decode):
+    """One key per (sequence, KV head) carries a logit far above the rest, so the softmax is an
+    exact one-hot in fp32: `out` must equal that key's V row bit for bit and the span masses are
+    exactly 1 / 0.  V rows are random, so any wrong page, slot, head or stride shows up."""
+    lens = [40, 700, 1300, 16, 129]
+    Hq, Hkv, D = 8, 2, 128
+    g = inputs._gen(404)
+    case = inputs.make_case("onehot", is_decode=decode, seq_lens=lens, q_lens=[1] * 5 if decode else [1, 3, 2, 1, 1],
+                            num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, seed=12, num_spans=2,
+                            head_mask=torch.ones(Hq, dtype=torch.uint8),
+                            probe_rows=inputs.PROBE_ROWS_LAST, poison=True)
+    case.q[:] = 4.0
+    hot = [int(torch.randint(0, L - 2 if not decode else L, (1,), generator=g)) for L in lens]
+    spans = torch.zeros((5, 2, 2), dtype=torch.int32)
+    for s, L in enumerate(lens):
+        pages = case.block_table[s, :(L + 15) // 16].long()
+        case.k_cache[pages] = torch.where(torch.isnan(case.k_cache[pages]), case.k_cache[pages], torch.zeros((), dtype=torch.bfloat16))
+        t = hot[s] if L > 2 else 0
+        hot[s] = t
+        case.k_cache[case.block_table[s, t // 16].item(), t % 16] = 4.0     # logit 4*4*128*scale = 181
+        spans[s, 0, 0], spans[s, 0, 1] = 0, t
+        spans[s, 1, 0], spans[s, 1, 1] = t, t + 1
+    case.spans = spans
+    out, mass, st = run_gpu(eng, case)
+    assert st == 0
+    cu = case.cu_q_lens.tolist()
+    for s in range(5):
+        t = hot[s]
+        vrow = case.v_cache[case.block_table[s, t // 16].item(), t % 16]        # [Hkv, D]
+        want = vrow.repeat_interleave(Hq // Hkv, dim=0)
+        last = cu[s + 1] - 1
+        # every row of the call that can see key t (the last row always can)
+        assert torch.equal(out[last].cpu().view(torch.int16), want.view(torch.int16)), f"seq {s}"
+        assert torch.all(mass[s, :, 0] == 0.0) and torch.all(mass[s, :, 1] == 1.0)
+
+
+def test_empty_batch_and_empty_sequences(eng):
+    case = inputs.make_case("empty_rows", is_decode=False, seq_lens=[40, 25], q_lens=[0, 0], num_q_heads=4,
+                            num_kv_heads=2, head_dim=64, seed=2)
+    out, mass, st = run_gpu(eng, case)
+    assert st == 0 and out.shape[0] == 0
+    p, _keep = binding.make_params(**{k: v for k, v in binding.case_to_device(
+        inputs.config2_decode(num_seqs=2, lo=5, hi=9)).items() if k not in ()})
+    p.num_seqs = 0
+    p.total_q = 0
+    assert eng.call(p, True) == binding.HOOK_ATTN_OK
+
+
+def test_device_detected_faults_set_the_status_word(eng):
+    """A block id outside the pool and a sequence longer than its table are refused by the kernels'
+    own bounds checks: no access is made, the status word carries the code."""
+    case = inputs.config2_decode(num_seqs=4, lo=100, hi=200)
+    bad = inputs.replace(case, block_table=case.block_table.clone())
+    bad.block_table[1, 2] = case.num_blocks + 5
+    _, _, st = run_gpu(eng, bad)
+    assert st == binding.HOOK_ATTN_ERR_BOUNDS
+    too_long = inputs.with_seq_lens(case, [case.max_blocks_per_seq * 16 + 1] + case.seq_lens.tolist()[1:])
+    out, _, st = run_gpu(eng, too_long)
+    assert st == binding.HOOK_ATTN_ERR_BOUNDS
+    assert torch.all(out[0] == 0)
+    pf = inputs.make_case("pf_bad", is_decode=False, seq_lens=[50], q_lens=[50], num_q_heads=4, num_kv_heads=2,
+                          head_dim=64, seed=3)
+    pf.block_table[0, 1] = -7
+    _, _, st = run_gpu(eng, pf)
+    assert st == binding.HOOK_ATTN_ERR_BOUNDS
+    more_rows_than_keys = inputs.replace(pf, seq_lens=torch.tensor([20], dtype=torch.int32),
+                                         block_table=inputs.make_case("x", is_decode=False, seq_lens=[50], q_lens=[50],
+                                                                      num_q_heads=4, num_kv_heads=2, head_dim=64,
+                                                                      seed=3).block_table)
+    _, _, st = run_gpu(eng, more_rows_than_keys)
+    assert st == binding.HOOK_ATTN_ERR_INVALID_ARG
+
+
+def test_strided_cache_views(eng):
+    """K/V given as views of a larger allocation (extra KV heads between the used ones)."""
+    case = inputs.config2_decode(num_seqs=6, lo=60, hi=500)
+    kw = binding.case_to_device(case)
+    nb, page, hkv, d = case.k_cache.shape
+    big_k = torch.full((nb, page, hkv + 3, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    big_v = torch.full_like(big_k, float("nan"))
+    big_k[:, :, 2:2 + hkv] = kw["k_cache"]
+    big_v[:, :, 2:2 + hkv] = kw["v_cache"]
+    out_ref, mass_ref, _ = run_gpu(eng, case)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    kw["k_cache"], kw["v_cache"] = big_k[:, :, 2:2 + hkv], big_v[:, :, 2:2 + hkv]
+    out, mass = eng.hook_attn_decode(status=status, **kw)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(out.view(torch.int16), out_ref.view(torch.int16)) and torch.equal(mass, mass_ref)
