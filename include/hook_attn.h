@@ -131,6 +131,31 @@ int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void*
  * bit-identical from run to run.  span_mass has one row per sequence. */
 int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
 
+/* Decode for callers that can neither allocate device memory nor hand over scratch.
+ * (The paper has no counterpart; this is a convenience of the library.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- a serving loop whose
+ * memory budget is already committed to the KV cache, a plug-in that only receives the hooked
+ * layer's tensors, or a latency-critical path where an allocation (and the synchronisation it
+ * implies) must never happen.  Such a caller cannot size and keep the `workspace` of
+ * hook_attn_decode, so here the split-K partials go into a fixed array of
+ * HOOK_ATTN_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the
+ * library holds that much memory until the process exits.
+ *
+ * Same arguments, outputs and results as hook_attn_decode; `workspace` and `workspace_bytes` are
+ * ignored.  The call allocates nothing and frees nothing.  A batch whose partials do not fit the
+ * array (hook_attn_workspace_bytes(p, 1) > HOOK_ATTN_STATIC_SCRATCH_BYTES) is refused with
+ * HOOK_ATTN_ERR_WORKSPACE and nothing is launched.  The handle's device must be the current
+ * device, otherwise HOOK_ATTN_ERR_INVALID_ARG.
+ *
+ * The first call on each device looks up the device address of the array; make that first call
+ * outside of any stream capture.  All calls on a device share the one array, which keeps whatever
+ * the previous call left in it: the kernels never read an entry they have not written in the
+ * same call, so nothing needs clearing -- but two calls whose work overlaps on the GPU (different
+ * streams, or concurrent host threads) race on it.  Issue them on one stream, or order them. */
+#define HOOK_ATTN_STATIC_SCRATCH_BYTES (16u << 20)
+int hook_attn_decode_static_scratch(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
+
 /* Human-readable name of a return / status code. */
 const char* hook_attn_strerror(int code);
 

@@ -26,7 +26,9 @@ HOOK_PROBE_ROWS_ALL = 0
 HOOK_PROBE_ROWS_LAST = 1
 
 EXPORTS = ("hook_attn_create", "hook_attn_destroy", "hook_attn_workspace_bytes",
-           "hook_attn_prefill", "hook_attn_decode", "hook_attn_strerror")
+           "hook_attn_prefill", "hook_attn_decode", "hook_attn_decode_static_scratch",
+           "hook_attn_strerror")
+STATIC_SCRATCH_BYTES = 16 << 20   # HOOK_ATTN_STATIC_SCRATCH_BYTES
 
 
 class HookAttnParams(ctypes.Structure):
@@ -74,7 +76,7 @@ def load_library() -> ctypes.CDLL:
         lib.hook_attn_destroy.argtypes = [ctypes.c_void_p]
         lib.hook_attn_workspace_bytes.restype = ctypes.c_size_t
         lib.hook_attn_workspace_bytes.argtypes = [ctypes.POINTER(HookAttnParams), ctypes.c_int]
-        for name in ("hook_attn_prefill", "hook_attn_decode"):
+        for name in ("hook_attn_prefill", "hook_attn_decode", "hook_attn_decode_static_scratch"):
             fn = getattr(lib, name)
             fn.restype = ctypes.c_int
             fn.argtypes = [ctypes.c_void_p, ctypes.POINTER(HookAttnParams), ctypes.c_void_p]
@@ -171,6 +173,15 @@ class HookAttn:
             stream = torch.cuda.current_stream(self.device).cuda_stream
         fn = self._lib.hook_attn_decode if is_decode else self._lib.hook_attn_prefill
         return int(fn(self._h, ctypes.byref(params), ctypes.c_void_p(stream)))
+
+    def call_decode_static_scratch(self, params: HookAttnParams, stream: Optional[int] = None) -> int:
+        """``hook_attn_decode_static_scratch``: decode for callers that cannot allocate or pass
+        scratch; the partials go into the library's fixed array (``STATIC_SCRATCH_BYTES``).
+        Returns the library's return code."""
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device).cuda_stream
+        return int(self._lib.hook_attn_decode_static_scratch(self._h, ctypes.byref(params),
+                                                             ctypes.c_void_p(stream)))
 
     # -- convenience ---------------------------------------------------------------------
     def plan(self, is_decode: bool, *, q, k_cache, v_cache, block_table, seq_lens, cu_q_lens=None,

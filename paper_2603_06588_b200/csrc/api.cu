@@ -2,6 +2,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace hook_attn {
@@ -173,6 +175,68 @@ int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* 
     if (!p->workspace || p->workspace_bytes < need) return HOOK_ATTN_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(p->workspace) & 15u) return HOOK_ATTN_ERR_WORKSPACE;
     if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    cudaError_t e = launch_decode(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
+}
+
+// ---- decode without any caller-provided or allocated scratch --------------------------------
+//
+// Some callers cannot allocate device memory at the point where they run attention: code inside
+// a memory-pool-managed serving loop that has handed its whole budget to the KV cache, plug-ins
+// that are only given the tensors of the layer they hook, and callers that must not trigger an
+// allocation (and the implicit synchronisation it brings) on their hot path.  For them the
+// split-K partials live in this fixed array, which every GPU that loads the library holds until
+// the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[HOOK_ATTN_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_ptr[kMaxDevices];   // device address of g_static_scratch, per device ordinal
+bool g_static_scratch_ready[kMaxDevices];
+std::mutex g_static_scratch_mutex;
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address: the
+// address the kernels can use has to be asked for, once per device, with that device current.
+int static_scratch_address(int device, float** out)
+{
+    if (device < 0 || device >= kMaxDevices) return HOOK_ATTN_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_ready[device]) {
+        void* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || ptr == nullptr) {
+            (void)cudaGetLastError();
+            return HOOK_ATTN_ERR_CUDA;
+        }
+        g_static_scratch_ptr[device] = static_cast<float*>(ptr);
+        g_static_scratch_ready[device] = true;
+    }
+    *out = g_static_scratch_ptr[device];
+    return HOOK_ATTN_OK;
+}
+}  // namespace
+
+int hook_attn_decode_static_scratch(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream)
+{
+    KernelArgs a;
+    HeadCfg hc;
+    int rc = prepare(p, true, a, hc);
+    if (rc != HOOK_ATTN_OK) return rc;
+    if (p->num_seqs > 0 && p->max_blocks_per_seq == 0) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (p->num_seqs == 0) return handle ? HOOK_ATTN_OK : HOOK_ATTN_ERR_INVALID_ARG;
+    a.chunk = decode_pick_chunk(p->num_seqs, p->num_kv_heads, p->max_blocks_per_seq, kDefaultSMs);
+    a.max_chunks = (p->max_blocks_per_seq * kPage + a.chunk - 1) / a.chunk;
+    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, a.max_chunks);
+    if (need > HOOK_ATTN_STATIC_SCRATCH_BYTES) return HOOK_ATTN_ERR_WORKSPACE;   // batch too large for the fixed array
+    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess) return HOOK_ATTN_ERR_CUDA;
+    if (current != handle->device) return HOOK_ATTN_ERR_INVALID_ARG;             // the handle's device must be current
+    float* scratch = nullptr;
+    rc = static_scratch_address(handle->device, &scratch);
+    if (rc != HOOK_ATTN_OK) return rc;
+    a.ws = scratch;   // every partial the merge reads is written by the split-K kernel of the same call:
+                      // nothing in the array has to start at zero, stale contents are never read
     cudaError_t e = launch_decode(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
 }
