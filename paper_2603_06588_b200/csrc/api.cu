@@ -1,5 +1,6 @@
 // C ABI of the hooked paged-attention library: argument validation, workspace sizing, dispatch.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -16,6 +17,10 @@ int decode_pick_chunk(int num_seqs, int Hkv, int max_blocks, int num_sms);
 cudaError_t configure_prefill_mma();
 cudaError_t launch_prefill_mma(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st);
 int prefill_mma_tiles_upper_bound(int total_q, int num_seqs);
+// prefill_tc.cu
+cudaError_t configure_prefill_tc();
+bool prefill_tc_supported(const KernelArgs& a, int head_dim);
+cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, cudaStream_t st);
 }  // namespace hook_attn
 
 using namespace hook_attn;
@@ -24,6 +29,7 @@ struct hook_attn_handle {
     int device;
     int num_sms;
     int cc_major, cc_minor;
+    bool prefer_tc;   // head_dim-128 prefill goes to the tcgen05 kernel (HOOK_ATTN_PREFILL_KERNEL=mma turns it off)
 };
 
 namespace {
@@ -121,6 +127,7 @@ int hook_attn_create(hook_attn_handle** handle, int device)
     if (cudaSetDevice(device) != cudaSuccess) return HOOK_ATTN_ERR_CUDA;
     cudaError_t e = configure_decode();
     if (e == cudaSuccess) e = configure_prefill_mma();
+    if (e == cudaSuccess) e = configure_prefill_tc();
     cudaSetDevice(prev);
     if (e != cudaSuccess) return HOOK_ATTN_ERR_CUDA;
     hook_attn_handle* h = new hook_attn_handle;
@@ -128,6 +135,8 @@ int hook_attn_create(hook_attn_handle** handle, int device)
     h->num_sms = prop.multiProcessorCount;
     h->cc_major = prop.major;
     h->cc_minor = prop.minor;
+    const char* pk = getenv("HOOK_ATTN_PREFILL_KERNEL");
+    h->prefer_tc = !(pk && strcmp(pk, "mma") == 0);
     *handle = h;
     return HOOK_ATTN_OK;
 }
@@ -156,8 +165,13 @@ int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void*
     if (rc != HOOK_ATTN_OK) return rc;
     if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
     if (p->num_seqs == 0 || p->total_q == 0) return HOOK_ATTN_OK;
-    a.total_tiles = prefill_mma_tiles_upper_bound(p->total_q, p->num_seqs);
-    cudaError_t e = launch_prefill_mma(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
+    cudaError_t e;
+    if (handle->prefer_tc && prefill_tc_supported(a, p->head_dim)) {
+        e = launch_prefill_tc(a, hc, static_cast<cudaStream_t>(cuda_stream));
+    } else {
+        a.total_tiles = prefill_mma_tiles_upper_bound(p->total_q, p->num_seqs);
+        e = launch_prefill_mma(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
+    }
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
 }
 

@@ -1,0 +1,663 @@
+// Prefill / chunked prefill of the hooked paged attention on the 5th-generation tensor cores
+// (head_dim 128): TMA-staged K/V pages, tcgen05.mma with accumulators in tensor memory.
+//
+// One CTA owns two consecutive 128-row query tiles ("A" and "B") of one (sequence, query head)
+// and walks the 128-key tiles they need.  Roles (10 warps):
+//   warps 0-3  softmax of tile A: one thread per query row, reads the scores S_A from tensor
+//              memory, keeps the online softmax and the span-mass accumulators, writes the bf16
+//              probabilities P_A back over S_A, rescales the output accumulator O_A when the
+//              running reference maximum moves, and runs the epilogue of tile A;
+//   warps 4-7  the same for tile B;
+//   warp  8    producer: resolves pages through the block table and issues one TMA box load per
+//              (page, 64-wide half of the head) into 128B-swizzled K and V stages;
+//   warp  9    owns tensor memory and issues the MMAs: S = Q K^T (both operands K-major in shared
+//              memory) and O += P V (P from tensor memory, V as the MN-major B operand), ordered
+//              PV(A,j) QK(A,j+1) PV(B,j) QK(B,j+1) so that one tile's softmax overlaps the other
+//              tile's tensor work.
+// Tensor memory (512 columns): S_A/P_A at 0, S_B/P_B at 128, O_A at 256, O_B at 384.
+//
+// The softmax keeps a *reference* maximum that is only raised when a tile's maximum exceeds it by
+// more than 2^8; probabilities, the running sum and the span accumulators all live in that frame,
+// so the result is exact (the reference cancels in o / l and s_j / l) while most tiles need no
+// rescale of the accumulator.  Span masses are added from the fp32 probabilities, before the
+// rounding to bf16: a key tile inside a span adds the tile's row sum, a tile that straddles a span
+// edge adds a masked row sum, a disjoint tile adds nothing.
+//
+// Every wait on an mbarrier is bounded; when one runs out the CTA reports HOOK_ATTN_ERR_TIMEOUT
+// through the status word, leaves its loops, releases tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace hook_attn {
+
+namespace tc {
+
+constexpr int kBM = 128;             // query rows per tile
+constexpr int kBN = 128;             // keys per tile
+constexpr int kHD = 128;             // head dim
+constexpr int kThreads = 320;
+constexpr int kProducerWarp = 8;
+constexpr int kMmaWarp = 9;
+constexpr int kTileBytes = kBM * kHD * 2;       // 32 KB: one Q, K or V tile
+constexpr int kHalfBytes = kTileBytes / 2;      // 16 KB: 128 rows x 64 elements
+constexpr int kStages = 2;
+constexpr int kSmemBytes = 2 * kTileBytes + 2 * kStages * kTileBytes + 1024;   // Q(A,B) + K,V stages + alignment slack
+constexpr uint32_t kTmemCols = 512;
+constexpr float kRescaleThreshold = 8.0f;       // log2 units
+
+// ---- mbarrier / TMA / tcgen05 wrappers --------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after about two seconds.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u && global_timer_ns() - t0 > 2000000000ull) return false;
+    }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const float (&v)[32])
+{
+    const uint32_t* r = reinterpret_cast<const uint32_t*>(v);
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; b_mn = 1 for an MN-major B operand.
+__host__ __device__ constexpr uint32_t instr_desc(uint32_t b_mn)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+struct Barriers {
+    uint64_t q_full[2];
+    uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+    uint64_t s_full[2], p_full[2], o_full[2];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+}  // namespace tc
+
+using namespace tc;
+
+template <int NS>
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ CUtensorMap map_q,
+                  const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ Barriers bars;
+    __shared__ int sh_span[2 * kMaxSpans];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = blockIdx.x;
+    const int kvh = h / a.G;
+
+    // ---- locate (sequence, pair of query tiles); later pairs of a sequence (more keys) come first ----
+    int t = blockIdx.y, s = 0, n = 0;
+    for (; s < a.num_seqs; ++s) {
+        n = a.cu_q_lens[s + 1] - a.cu_q_lens[s];
+        const int np = (n + 2 * kBM - 1) / (2 * kBM);
+        if (t < np) { t = np - 1 - t; break; }
+        t -= np;
+    }
+    if (s >= a.num_seqs) return;
+    // once any CTA of this launch has given up on a wait, the rest of the grid does not start
+    if (a.status && *reinterpret_cast<volatile int32_t*>(a.status) == HOOK_ATTN_ERR_TIMEOUT) return;
+    const int L = a.seq_lens[s];
+    const int64_t grow_seq = a.cu_q_lens[s];
+    const int row0[2] = {2 * t * kBM, (2 * t + 1) * kBM};
+    int rows[2], first_pos[2], ntiles[2];
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+        rows[x] = max(0, min(kBM, n - row0[x]));
+        first_pos[x] = L - n + row0[x];
+        ntiles[x] = rows[x] > 0 ? (first_pos[x] + rows[x] - 1) / kBN + 1 : 0;
+    }
+    if (n > L || L > a.max_blocks * kPage) {
+        if (threadIdx.x == 0) report(a.status, n > L ? HOOK_ATTN_ERR_INVALID_ARG : HOOK_ATTN_ERR_BOUNDS);
+        const int nrows = rows[0] + rows[1];
+        for (int idx = threadIdx.x; idx < nrows * kHD; idx += kThreads)
+            a.out[((grow_seq + row0[0] + idx / kHD) * a.Hq + h) * kHD + idx % kHD] = __float2bfloat16(0.f);
+        return;
+    }
+    const int nmax = max(ntiles[0], ntiles[1]);
+    const int slot = (NS > 0) ? hc.slot[h] : -1;
+    const bool probe = (NS > 0) && slot >= 0;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t sQ[2] = {smem_base, smem_base + kTileBytes};
+    const uint32_t sK = smem_base + 2 * kTileBytes;
+    const uint32_t sV = sK + kStages * kTileBytes;
+
+    // ---- set-up: barriers, spans, tensor memory ----
+    if (threadIdx.x == 0) {
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(smem_u32(&bars.q_full[x]), 1);
+            mbar_init(smem_u32(&bars.s_full[x]), 1);
+            mbar_init(smem_u32(&bars.p_full[x]), 128);
+            mbar_init(smem_u32(&bars.o_full[x]), 1);
+        }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(smem_u32(&bars.k_full[i]), 1);
+            mbar_init(smem_u32(&bars.k_empty[i]), 1);
+            mbar_init(smem_u32(&bars.v_full[i]), 1);
+            mbar_init(smem_u32(&bars.v_empty[i]), 1);
+        }
+        bars.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (NS > 0 && (int)threadIdx.x < 2 * NS) {
+        const int j = threadIdx.x >> 1;
+        sh_span[threadIdx.x] = (probe && j < a.S) ? a.spans[((int64_t)s * a.S + j) * 2 + (threadIdx.x & 1)] : 0;
+    }
+    if (warp == kMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars.tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = bars.tmem_base;
+    bool ok = true;   // false once a bounded wait ran out
+
+    if (warp == kProducerWarp) {
+        // ================================ producer ================================
+        const int32_t* bt = a.block_table + (int64_t)s * a.max_blocks;
+        if (lane == 0) {
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                if (ntiles[x] > 0) {
+                    const uint32_t bar = smem_u32(&bars.q_full[x]);
+                    mbar_expect_tx(bar, kTileBytes);
+                    tma_load_3d(sQ[x], &map_q, bar, 0, h, (int)(grow_seq + row0[x]));
+                    tma_load_3d(sQ[x] + kHalfBytes, &map_q, bar, 64, h, (int)(grow_seq + row0[x]));
+                }
+            }
+        }
+        for (int j = 0; j < nmax && ok; ++j) {
+            const int st = j & 1;
+            const uint32_t ph = (j >> 1) & 1;
+            const int pages = min(kBN / kPage, (L - j * kBN + kPage - 1) / kPage);   // pages that hold keys < L
+            int blk = 0;
+            const int pg = lane >> 1, half = lane & 1;
+            if (lane < 16 && pg < pages) {
+                blk = bt[j * (kBN / kPage) + pg];
+                if (blk < 0 || blk >= a.num_blocks) { report(a.status, HOOK_ATTN_ERR_BOUNDS); blk = 0; }
+            }
+#pragma unroll
+            for (int kv = 0; kv < 2; ++kv) {
+                const uint32_t full = smem_u32(kv ? &bars.v_full[st] : &bars.k_full[st]);
+                const uint32_t empty = smem_u32(kv ? &bars.v_empty[st] : &bars.k_empty[st]);
+                ok = __all_sync(0xffffffffu, mbar_wait(empty, ph ^ 1u));
+                if (!ok) break;
+                if (lane == 0) mbar_expect_tx(full, (uint32_t)pages * 2u * (kPage * 128u));
+                __syncwarp();
+                if (lane < 16 && pg < pages) {
+                    const uint32_t dst = (kv ? sV : sK) + st * kTileBytes + half * kHalfBytes + pg * (kPage * 128);
+                    tma_load_4d(dst, kv ? &map_v : &map_k, full, half * 64, kvh, 0, blk);
+                }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ================================ MMA issue ================================
+        constexpr uint32_t idesc_qk = instr_desc(0), idesc_pv = instr_desc(1);
+        const uint32_t tS[2] = {tmem, tmem + 128}, tO[2] = {tmem + 256, tmem + 384};
+        auto issue_qk = [&](int x, int j) {
+            const uint32_t kb = sK + (j & 1) * kTileBytes;
+#pragma unroll
+            for (int ks = 0; ks < kHD / 16; ++ks) {
+                const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+                tc_mma_ss(tS[x], smem_desc(sQ[x] + off, 16, 1024), smem_desc(kb + off, 16, 1024), idesc_qk, ks > 0);
+            }
+            tc_commit(smem_u32(&bars.s_full[x]));
+        };
+        auto issue_pv = [&](int x, int j) {
+            const uint32_t vb = sV + (j & 1) * kTileBytes;
+#pragma unroll
+            for (int ks = 0; ks < kBN / 16; ++ks)
+                tc_mma_ts(tO[x], tS[x] + ks * 8, smem_desc(vb + ks * (16 * 128), kHalfBytes, 1024), idesc_pv, (j > 0) || (ks > 0));
+        };
+#pragma unroll
+        for (int x = 0; x < 2; ++x)
+            if (ok && ntiles[x] > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full[x]), 0));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.k_full[0]), 0));
+        if (ok) {
+            tc_fence_after();
+            if (lane == 0) {
+                if (ntiles[0] > 0) issue_qk(0, 0);
+                if (ntiles[1] > 0) issue_qk(1, 0);
+                if (kStages < nmax) tc_commit(smem_u32(&bars.k_empty[0]));   // only if the producer will wait for it
+            }
+            __syncwarp();
+        }
+        for (int j = 0; j < nmax && ok; ++j) {
+            const int st = j & 1;
+            const uint32_t ph = (j >> 1) & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_full[st]), ph));
+            if (!ok) break;
+            if (j == nmax - 1 && (j + 1) * kBN > L) {
+                // value rows at keys >= L (page tails, pages that were never loaded) must not reach the
+                // tensor cores: 0 * NaN would poison the accumulator.  Zero them in shared memory.
+                const int r_first = L - j * kBN;
+                const uint32_t vb = sV + st * kTileBytes;
+                for (int idx = lane; idx < (kBN - r_first) * 16; idx += 32) {
+                    const int r = r_first + (idx >> 4), c = idx & 15;
+                    const uint32_t addr = vb + (c >> 3) * kHalfBytes + r * 128 + (c & 7) * 16;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+            }
+            const bool has_next = (j + 1 < nmax);
+            if (has_next) {
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.k_full[(j + 1) & 1]), ((j + 1) >> 1) & 1));
+                if (!ok) break;
+            }
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                if (j < ntiles[x]) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.p_full[x]), j & 1));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        issue_pv(x, j);
+                        if (j + 1 < ntiles[x]) issue_qk(x, j + 1);
+                        else tc_commit(smem_u32(&bars.o_full[x]));
+                    }
+                    __syncwarp();
+                }
+            }
+            if (!ok) break;
+            if (lane == 0) {
+                // release a stage only if the producer will refill it: an arrive that nobody waits for
+                // could land after the CTA has gone
+                if (j + kStages < nmax) tc_commit(smem_u32(&bars.v_empty[st]));
+                if (j + 1 + kStages < nmax) tc_commit(smem_u32(&bars.k_empty[(j + 1) & 1]));
+            }
+            __syncwarp();
+        }
+    } else {
+        // ================================ softmax + epilogue ================================
+        const int x = warp >> 2;                      // 0 = tile A, 1 = tile B
+        const int nt = ntiles[x];
+        if (nt > 0) {
+            const int quarter = warp & 3;
+            const int row = quarter * 32 + lane;
+            const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+            const uint32_t tS = tmem + x * 128 + lane_off;
+            const uint32_t tO = tmem + 256 + x * 128 + lane_off;
+            const int pos = min(first_pos[x] + row, L - 1);
+            const float sl2 = a.scale_log2;
+            float m_ref = -INFINITY, l = 0.f;
+            float sm[NS > 0 ? NS : 1];
+#pragma unroll
+            for (int js = 0; js < (NS > 0 ? NS : 1); ++js) sm[js] = 0.f;
+
+            for (int j = 0; j < nt && ok; ++j) {
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), j & 1));
+                if (!ok) break;
+                tc_fence_after();
+                const int k0 = j * kBN;
+                const bool need_mask = (k0 + kBN - 1 > first_pos[x]);
+                float v[32];
+
+                // pass 1: row maximum of the visible scores
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    tc_ld32(tS + 32 * c, v);
+                    tc_wait_ld();
+                    if (need_mask) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (k0 + 32 * c + i <= pos) ? v[i] : -INFINITY);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, v[i]);
+                    }
+                }
+                mx *= sl2;
+                // raise the reference maximum only when it is exceeded by more than the threshold
+                const bool raise = mx > m_ref + kRescaleThreshold;
+                if (__any_sync(0xffffffffu, raise)) {
+                    const float m_new = fmaxf(m_ref, mx);
+                    const float f = (m_ref == -INFINITY) ? 0.f : fast_exp2(m_ref - m_new);
+                    m_ref = m_new;
+                    l *= f;
+#pragma unroll
+                    for (int js = 0; js < (NS > 0 ? NS : 1); ++js) sm[js] *= f;
+                    if (j > 0) {
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            tc_ld32(tO + 32 * c, v);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] *= f;
+                            tc_st32(tO + 32 * c, v);
+                        }
+                        tc_wait_st();
+                    }
+                }
+
+                // which spans does this key tile touch?
+                uint32_t full_mask = 0, part_mask = 0;
+                if (NS > 0 && probe) {
+#pragma unroll
+                    for (int js = 0; js < NS; ++js) {
+                        const int sa = sh_span[2 * js], sb = sh_span[2 * js + 1];
+                        if (sb > k0 && sa < k0 + kBN) {
+                            if (sa <= k0 && sb >= k0 + kBN) full_mask |= 1u << js; else part_mask |= 1u << js;
+                        }
+                    }
+                }
+
+                // pass 2: probabilities (fp32 sums, bf16 for the tensor cores), written over S
+                const float neg_m = -m_ref;
+                float rs = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    tc_ld32(tS + 32 * c, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        float p = fast_exp2(fmaf(v[i], sl2, neg_m));
+                        if (need_mask && (k0 + 32 * c + i > pos)) p = 0.f;
+                        v[i] = p;
+                        rs += p;
+                    }
+                    if (NS > 0 && part_mask) {
+#pragma unroll
+                        for (int js = 0; js < NS; ++js) {
+                            if (part_mask & (1u << js)) {
+                                const int sa = sh_span[2 * js], sb = sh_span[2 * js + 1];
+                                float acc = 0.f;
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) {
+                                    const int key = k0 + 32 * c + i;
+                                    acc += (key >= sa && key < sb) ? v[i] : 0.f;
+                                }
+                                sm[js] += acc;
+                            }
+                        }
+                    }
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
+                    tc_st16(tS + 16 * c, pk);
+                }
+                tc_wait_st();
+                l += rs;
+                if (NS > 0 && full_mask) {
+#pragma unroll
+                    for (int js = 0; js < NS; ++js)
+                        if (full_mask & (1u << js)) sm[js] += rs;
+                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars.p_full[x]));
+            }
+
+            // ---- epilogue: normalise, steer, round once, store ----
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_full[x]), 0));
+            if (ok) {
+                tc_fence_after();
+                const float inv = 1.f / l;
+                const float al = hc.alpha[h];
+                const float* sv = a.steer + (int64_t)h * kHD;
+                const bool live = row < rows[x];
+                __nv_bfloat16* orow = a.out + ((grow_seq + row0[x] + row) * a.Hq + h) * kHD;
+                float v[32];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    tc_ld32(tO + 32 * c, v);
+                    tc_wait_ld();
+                    if (live) {
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int d = 32 * c + 8 * q4 + 2 * i;
+                                float y0 = v[8 * q4 + 2 * i] * inv, y1 = v[8 * q4 + 2 * i + 1] * inv;
+                                if (al != 0.f) { y0 = fmaf(al, sv[d], y0); y1 = fmaf(al, sv[d + 1], y1); }
+                                w[i] = pack_bf16(y0, y1);
+                            }
+                            *reinterpret_cast<uint4*>(orow + 32 * c + 8 * q4) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                }
+                if (NS > 0 && probe && live) {
+                    const bool last_only = (a.probe_rows == HOOK_PROBE_ROWS_LAST);
+                    if (!last_only || row0[x] + row == n - 1) {
+                        const int64_t mrow = last_only ? (int64_t)s : grow_seq + row0[x] + row;
+                        float* dst = a.mass + (mrow * a.P + slot) * a.S;
+#pragma unroll
+                        for (int js = 0; js < NS; ++js)
+                            if (js < a.S) dst[js] = sm[js] * inv;
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown ----
+    if (!ok) {
+        if (lane == 0) report(a.status, HOOK_ATTN_ERR_TIMEOUT);
+        atomicExch(&bars.abort_flag, 1);
+        const uint64_t t0 = global_timer_ns();           // let copies that are still in flight land
+        while (global_timer_ns() - t0 < 1000000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            (void)cudaGetLastError();
+    }
+    return fn;
+}
+
+bool encode(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+            const cuuint32_t* box)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box, ones,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int NS>
+cudaError_t launch_t(const KernelArgs& a, const HeadCfg& hc, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                     int pairs, cudaStream_t st)
+{
+    prefill_tc_kernel<NS><<<dim3(a.Hq, pairs), kThreads, kSmemBytes, st>>>(a, hc, mq, mk, mv);
+    return cudaGetLastError();
+}
+
+template <int NS>
+cudaError_t configure_one()
+{
+    return cudaFuncSetAttribute(prefill_tc_kernel<NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
+}  // namespace
+
+cudaError_t configure_prefill_tc()
+{
+    cudaError_t e;
+    if ((e = configure_one<0>()) != cudaSuccess) return e;
+    if ((e = configure_one<2>()) != cudaSuccess) return e;
+    if ((e = configure_one<4>()) != cudaSuccess) return e;
+    return configure_one<8>();
+}
+
+// True when the tensor-core kernel can serve the call (head_dim 128, tensor maps encodable).
+bool prefill_tc_supported(const KernelArgs& a, int head_dim)
+{
+    return head_dim == kHD && a.total_q >= kBM && a.num_blocks > 0 && encode_fn() != nullptr &&
+           a.bs < (1ll << 38) && a.ts < (1ll << 38) && a.hs < (1ll << 38);
+}
+
+cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, cudaStream_t st)
+{
+    CUtensorMap mq, mk, mv;
+    {
+        const cuuint64_t dims[3] = {(cuuint64_t)kHD, (cuuint64_t)a.Hq, (cuuint64_t)a.total_q};
+        const cuuint64_t strides[2] = {(cuuint64_t)kHD * 2, (cuuint64_t)a.Hq * kHD * 2};
+        const cuuint32_t box[3] = {64, 1, (cuuint32_t)kBM};
+        if (!encode(&mq, a.q, 3, dims, strides, box)) return cudaErrorInvalidValue;
+    }
+    {
+        const cuuint64_t dims[4] = {(cuuint64_t)kHD, (cuuint64_t)a.Hkv, (cuuint64_t)kPage, (cuuint64_t)a.num_blocks};
+        const cuuint64_t strides[3] = {(cuuint64_t)a.hs * 2, (cuuint64_t)a.ts * 2, (cuuint64_t)a.bs * 2};
+        const cuuint32_t box[4] = {64, 1, (cuuint32_t)kPage, 1};
+        if (!encode(&mk, a.k, 4, dims, strides, box)) return cudaErrorInvalidValue;
+        if (!encode(&mv, a.v, 4, dims, strides, box)) return cudaErrorInvalidValue;
+    }
+    // sum over sequences of ceil(n_s / 256) <= floor(total_q / 256) + num_seqs
+    const int pairs = a.total_q / (2 * kBM) + a.num_seqs;
+    const int ns = !a.any_probe ? 0 : (a.S <= 2 ? 2 : (a.S <= 4 ? 4 : 8));
+    switch (ns) {
+        case 0: return launch_t<0>(a, hc, mq, mk, mv, pairs, st);
+        case 2: return launch_t<2>(a, hc, mq, mk, mv, pairs, st);
+        case 4: return launch_t<4>(a, hc, mq, mk, mv, pairs, st);
+        default: return launch_t<8>(a, hc, mq, mk, mv, pairs, st);
+    }
+}
+
+}  // namespace hook_attn
