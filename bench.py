@@ -40,6 +40,7 @@ UNIT = "tokens/s"
 WORKLOADS = {
     "cfg2_decode": "decode batch: 64 seqs x 1 token, ctx U[512,4096], Hq32/Hkv8, D128, 16 probed heads, 2 spans, 4 steered heads",
     "cfg3_prefill": "prefill: 8 seqs x 4096 tokens causal, Hq32/Hkv8, D128, ~10% (layer,head) pairs probed, 3 spans, one layer call per step",
+    "cfg3_prefill_small": "prefill, profiling size: 2 seqs x 2048 tokens causal, Hq32/Hkv8, D128, layer-0 probes, 3 spans",
     "cfg4_decode": "mixed batch, decode part: 256 seqs, ctx U[1024,8192], Hq28/Hkv4, D128, 14 probed heads, 4 spans, 8 steered heads",
     "cfg4_prefill": "mixed batch, prefill part: 2 chunks of 2048 tokens on 4096-token contexts, Hq28/Hkv4, D128",
     "cfg5_decode": "long context decode: 4 seqs at 32768+ keys, Hq64/Hkv8, D128, 64 probed heads, 8 spans, 8 steered heads",
@@ -52,6 +53,8 @@ def make_workload(name: str):
         return inputs.config2_decode()
     if name == "cfg3_prefill":
         return inputs.config3_prefill(layer=0, force_probe=True)
+    if name == "cfg3_prefill_small":
+        return inputs.config3_prefill(layer=0, num_seqs=2, tokens=2048, force_probe=True)
     if name == "cfg4_decode":
         return inputs.config4_decode()
     if name == "cfg4_prefill":

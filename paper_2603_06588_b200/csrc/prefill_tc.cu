@@ -2,7 +2,7 @@
 // (head_dim 128): TMA-staged K/V pages, tcgen05.mma with accumulators in tensor memory.
 //
 // One CTA owns two consecutive 128-row query tiles ("A" and "B") of one (sequence, query head)
-// and walks the 128-key tiles they need.  Roles (10 warps):
+// and walks the 128-key tiles they need.  Roles (12 warps, three warpgroups):
 //   warps 0-3  softmax of tile A: one thread per query row, reads the scores S_A from tensor
 //              memory, keeps the online softmax and the span-mass accumulators, writes the bf16
 //              probabilities P_A back over S_A, rescales the output accumulator O_A when the
@@ -36,7 +36,7 @@ namespace tc {
 constexpr int kBM = 128;             // query rows per tile
 constexpr int kBN = 128;             // keys per tile
 constexpr int kHD = 128;             // head dim
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;            // three warpgroups: softmax A, softmax B, {producer, MMA, 2 idle warps}
 constexpr int kProducerWarp = 8;
 constexpr int kMmaWarp = 9;
 constexpr int kTileBytes = kBM * kHD * 2;       // 32 KB: one Q, K or V tile
@@ -45,6 +45,19 @@ constexpr int kStages = 2;
 constexpr int kSmemBytes = 2 * kTileBytes + 2 * kStages * kTileBytes + 1024;   // Q(A,B) + K,V stages + alignment slack
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;       // log2 units
+constexpr int kMaskTiles = 1024;                // key tiles with a precomputed span classification
+
+// Which spans does key tile [k0, k0 + 128) touch?  Low byte: spans that contain the whole tile;
+// high byte: spans that straddle it (their masked row sum is needed).
+__device__ __forceinline__ uint32_t classify_tile(const int* span, int ns, int k0)
+{
+    uint32_t m = 0;
+    for (int js = 0; js < ns; ++js) {
+        const int sa = span[2 * js], sb = span[2 * js + 1];
+        if (sb > k0 && sa < k0 + kBN && sb > sa) m |= (sa <= k0 && sb >= k0 + kBN) ? (1u << js) : (0x100u << js);
+    }
+    return m;
+}
 
 // ---- mbarrier / TMA / tcgen05 wrappers --------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
@@ -127,7 +140,7 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t bdesc
         ::"r"(d), "r"(a), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32])
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v)   // v: 32 consecutive values (registers)
 {
     uint32_t* r = reinterpret_cast<uint32_t*>(v);
     asm volatile(
@@ -154,7 +167,7 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const float (&v)[32])
           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
-__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16])
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r)   // r: 16 consecutive values (registers)
 {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -164,6 +177,25 @@ __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16])
         : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Wait for outstanding tensor-memory loads and tie the 32 loaded values to the wait, so that no use
+// of them can be scheduled ahead of it.
+__device__ __forceinline__ void tc_wait_ld_dep(float* v)
+{
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                   "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                   "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
@@ -171,6 +203,11 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 {
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
            (1ull << 46) | (2ull << 61);
+}
+// Move the start-address field (units of 16 bytes) of a descriptor; the field never overflows here.
+__device__ __forceinline__ uint64_t desc_advance(uint64_t d, uint32_t units16)
+{
+    return ((uint64_t)(uint32_t)(d >> 32) << 32) | (uint64_t)((uint32_t)d + units16);
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, M = 128, N = 128; b_mn = 1 for an MN-major B operand.
 __host__ __device__ constexpr uint32_t instr_desc(uint32_t b_mn)
@@ -198,6 +235,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
     extern __shared__ uint8_t smem_raw[];
     __shared__ Barriers bars;
     __shared__ int sh_span[2 * kMaxSpans];
+    __shared__ uint16_t sh_tile_mask[kMaskTiles];   // per key tile: bits 0-7 spans covering it, bits 8-15 spans straddling it
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.x;
@@ -261,6 +299,11 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
         const int j = threadIdx.x >> 1;
         sh_span[threadIdx.x] = (probe && j < a.S) ? a.spans[((int64_t)s * a.S + j) * 2 + (threadIdx.x & 1)] : 0;
     }
+    if (NS > 0 && probe) {
+        const int* gspan = a.spans + (int64_t)s * a.S * 2;
+        for (int jj = threadIdx.x; jj < min(nmax, kMaskTiles); jj += kThreads)
+            sh_tile_mask[jj] = (uint16_t)classify_tile(gspan, a.S, jj * kBN);
+    }
     if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars.tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -271,6 +314,15 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
     const uint32_t tmem = bars.tmem_base;
     bool ok = true;   // false once a bounded wait ran out
 
+    // Register split between the warpgroups: the softmax threads keep a whole 128-wide score row in
+    // registers, the producer/MMA warpgroup needs few.  Launched with 168 per thread (384 x 168 =
+    // 64512); after the split 128 x (208 + 208 + 72) = 62464, which fits the launch allocation.
+
+
+
+    if (warp >= 8) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;" ::: "memory");
+    }
     if (warp == kProducerWarp) {
         // ================================ producer ================================
         const int32_t* bt = a.block_table + (int64_t)s * a.max_blocks;
@@ -313,20 +365,25 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
         // ================================ MMA issue ================================
         constexpr uint32_t idesc_qk = instr_desc(0), idesc_pv = instr_desc(1);
         const uint32_t tS[2] = {tmem, tmem + 128}, tO[2] = {tmem + 256, tmem + 384};
+        // Descriptors are built once; per MMA only the start-address field moves (one 32-bit add), so
+        // that the single issuing thread keeps the tensor pipe fed.
+        const uint64_t dQ[2] = {smem_desc(sQ[0], 16, 1024), smem_desc(sQ[1], 16, 1024)};
+        const uint64_t dK[2] = {smem_desc(sK, 16, 1024), smem_desc(sK + kTileBytes, 16, 1024)};
+        const uint64_t dV[2] = {smem_desc(sV, kHalfBytes, 1024), smem_desc(sV + kTileBytes, kHalfBytes, 1024)};
         auto issue_qk = [&](int x, int j) {
-            const uint32_t kb = sK + (j & 1) * kTileBytes;
+            const uint64_t dq = dQ[x], dk = (j & 1) ? dK[1] : dK[0];
 #pragma unroll
             for (int ks = 0; ks < kHD / 16; ++ks) {
-                const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                tc_mma_ss(tS[x], smem_desc(sQ[x] + off, 16, 1024), smem_desc(kb + off, 16, 1024), idesc_qk, ks > 0);
+                const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+                tc_mma_ss(tS[x], desc_advance(dq, off), desc_advance(dk, off), idesc_qk, ks > 0);
             }
             tc_commit(smem_u32(&bars.s_full[x]));
         };
         auto issue_pv = [&](int x, int j) {
-            const uint32_t vb = sV + (j & 1) * kTileBytes;
+            const uint64_t dv = (j & 1) ? dV[1] : dV[0];
 #pragma unroll
             for (int ks = 0; ks < kBN / 16; ++ks)
-                tc_mma_ts(tO[x], tS[x] + ks * 8, smem_desc(vb + ks * (16 * 128), kHalfBytes, 1024), idesc_pv, (j > 0) || (ks > 0));
+                tc_mma_ts(tO[x], tS[x] + ks * 8, desc_advance(dv, (ks * 16 * 128) >> 4), idesc_pv, (ks > 0) || (j > 0));
         };
 #pragma unroll
         for (int x = 0; x < 2; ++x)
@@ -387,7 +444,8 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             }
             __syncwarp();
         }
-    } else {
+    } else if (warp < 8) {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;" ::: "memory");
         // ================================ softmax + epilogue ================================
         const int x = warp >> 2;                      // 0 = tile A, 1 = tile B
         const int nt = ntiles[x];
@@ -410,23 +468,32 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
                 tc_fence_after();
                 const int k0 = j * kBN;
                 const bool need_mask = (k0 + kBN - 1 > first_pos[x]);
-                float v[32];
 
-                // pass 1: row maximum of the visible scores
-                float mx = -INFINITY;
+                uint32_t tm = 0;   // spans touching this key tile: low byte covering, high byte straddling
+                if (NS > 0 && probe) tm = (j < kMaskTiles) ? sh_tile_mask[j] : classify_tile(sh_span, NS, k0);
+
+                // the whole score row of this thread: four loads in flight, one wait
+                float sc[kBN];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    tc_ld32(tS + 32 * c, v);
-                    tc_wait_ld();
-                    if (need_mask) {
+                for (int c = 0; c < 4; ++c) tc_ld32(tS + 32 * c, sc + 32 * c);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (k0 + 32 * c + i <= pos) ? v[i] : -INFINITY);
-                    } else {
+                for (int c = 0; c < 4; ++c) tc_wait_ld_dep(sc + 32 * c);
+                if (need_mask) {
+                    // causal / end-of-sequence mask as a select (stale or poisoned keys never propagate)
+                    const int lim = pos - k0;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, v[i]);
-                    }
+                    for (int i = 0; i < kBN; ++i) sc[i] = (i <= lim) ? sc[i] : -INFINITY;
                 }
-                mx *= sl2;
+                float mxp[4];   // four independent chains keep the dependency depth short
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    float t = max3(sc[32 * q4], sc[32 * q4 + 1], sc[32 * q4 + 2]);
+#pragma unroll
+                    for (int i = 3; i + 1 < 32; i += 2) t = max3(t, sc[32 * q4 + i], sc[32 * q4 + i + 1]);
+                    mxp[q4] = fmaxf(t, sc[32 * q4 + 31]);
+                }
+                const float mx = fmaxf(max3(mxp[0], mxp[1], mxp[2]), mxp[3]) * sl2;
+
                 // raise the reference maximum only when it is exceeded by more than the threshold
                 const bool raise = mx > m_ref + kRescaleThreshold;
                 if (__any_sync(0xffffffffu, raise)) {
@@ -437,10 +504,11 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
 #pragma unroll
                     for (int js = 0; js < (NS > 0 ? NS : 1); ++js) sm[js] *= f;
                     if (j > 0) {
+                        float v[32];
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             tc_ld32(tO + 32 * c, v);
-                            tc_wait_ld();
+                            tc_wait_ld_dep(v);
 #pragma unroll
                             for (int i = 0; i < 32; ++i) v[i] *= f;
                             tc_st32(tO + 32 * c, v);
@@ -449,59 +517,61 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
                     }
                 }
 
-                // which spans does this key tile touch?
-                uint32_t full_mask = 0, part_mask = 0;
-                if (NS > 0 && probe) {
-#pragma unroll
-                    for (int js = 0; js < NS; ++js) {
-                        const int sa = sh_span[2 * js], sb = sh_span[2 * js + 1];
-                        if (sb > k0 && sa < k0 + kBN) {
-                            if (sa <= k0 && sb >= k0 + kBN) full_mask |= 1u << js; else part_mask |= 1u << js;
-                        }
-                    }
-                }
-
-                // pass 2: probabilities (fp32 sums, bf16 for the tensor cores), written over S
-                const float neg_m = -m_ref;
-                float rs = 0.f;
+                // probabilities in the frame of the reference maximum: fp32 for the sums, bf16 pairs
+                // written over the scores for the tensor cores
+                const float2 sl2v = make_float2(sl2, sl2), nmv = make_float2(-m_ref, -m_ref);
+                float2 rs2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    tc_ld32(tS + 32 * c, v);
-                    tc_wait_ld();
+                    uint32_t pk[16];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        float p = fast_exp2(fmaf(v[i], sl2, neg_m));
-                        if (need_mask && (k0 + 32 * c + i > pos)) p = 0.f;
-                        v[i] = p;
-                        rs += p;
+                    for (int i = 0; i < 16; ++i) {
+                        const int e = 32 * c + 2 * i;
+                        const float2 xx = __ffma2_rn(make_float2(sc[e], sc[e + 1]), sl2v, nmv);
+                        const float2 pp = make_float2(fast_exp2(xx.x), fast_exp2(xx.y));
+                        sc[e] = pp.x;
+                        sc[e + 1] = pp.y;
+                        rs2[i & 1] = __fadd2_rn(rs2[i & 1], pp);
+                        pk[i] = pack_bf16(pp.x, pp.y);
                     }
-                    if (NS > 0 && part_mask) {
+                    tc_st16(tS + 16 * c, pk);
+                }
+                const float rs = (rs2[0].x + rs2[0].y) + (rs2[1].x + rs2[1].y);
+                l += rs;
+
+                // span masses: a tile inside a span adds the row sum, a straddling tile a masked sum
+                if (NS > 0 && probe) {
+                    if (tm & 0xffu) {
 #pragma unroll
+                        for (int js = 0; js < NS; ++js) sm[js] += ((tm >> js) & 1u) ? rs : 0.f;
+                    }
+                    if (tm & 0xff00u) {
+#pragma unroll 1
                         for (int js = 0; js < NS; ++js) {
-                            if (part_mask & (1u << js)) {
-                                const int sa = sh_span[2 * js], sb = sh_span[2 * js + 1];
-                                float acc = 0.f;
+                            if (!((tm >> (8 + js)) & 1u)) continue;
+                            const int lo = sh_span[2 * js] - k0, hi = sh_span[2 * js + 1] - k0;
+                            const uint32_t width = (uint32_t)(hi - lo);
+                            float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) {
-                                    const int key = k0 + 32 * c + i;
-                                    acc += (key >= sa && key < sb) ? v[i] : 0.f;
-                                }
-                                sm[js] += acc;
+                            for (int i = 0; i < kBN; i += 2) {
+                                acc0 += ((uint32_t)(i - lo) < width) ? sc[i] : 0.f;
+                                acc1 += ((uint32_t)(i + 1 - lo) < width) ? sc[i + 1] : 0.f;
+                            }
+                            const float add = acc0 + acc1;
+                            switch (js) {   // static register targets
+                                case 0: sm[0] += add; break;
+                                case 1: if (NS > 1) sm[NS > 1 ? 1 : 0] += add; break;
+                                case 2: if (NS > 2) sm[NS > 2 ? 2 : 0] += add; break;
+                                case 3: if (NS > 3) sm[NS > 3 ? 3 : 0] += add; break;
+                                case 4: if (NS > 4) sm[NS > 4 ? 4 : 0] += add; break;
+                                case 5: if (NS > 5) sm[NS > 5 ? 5 : 0] += add; break;
+                                case 6: if (NS > 6) sm[NS > 6 ? 6 : 0] += add; break;
+                                default: if (NS > 7) sm[NS > 7 ? 7 : 0] += add; break;
                             }
                         }
                     }
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(v[2 * i], v[2 * i + 1]);
-                    tc_st16(tS + 16 * c, pk);
                 }
                 tc_wait_st();
-                l += rs;
-                if (NS > 0 && full_mask) {
-#pragma unroll
-                    for (int js = 0; js < NS; ++js)
-                        if (full_mask & (1u << js)) sm[js] += rs;
-                }
                 tc_fence_before();
                 mbar_arrive(smem_u32(&bars.p_full[x]));
             }
@@ -519,7 +589,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     tc_ld32(tO + 32 * c, v);
-                    tc_wait_ld();
+                    tc_wait_ld_dep(v);
                     if (live) {
 #pragma unroll
                         for (int q4 = 0; q4 < 4; ++q4) {
