@@ -10,7 +10,7 @@
 // sum.  The four warps are merged in shared memory and the chunk's partial (m, l, o[D], s[S]) is
 // written to the workspace.
 //
-// Kernel 2 (decode_merge): one CTA per (query head, sequence) merges the chunk partials in chunk
+// Kernel 2 (decode_merge): one CTA per (query head, sequence) merges the chunk partials in a fixed
 // order (run-to-run bit-identical), normalises, applies the steering add and stores.
 #include "common.cuh"
 
@@ -247,21 +247,32 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_splitk_kernel(const Ker
     }
 }
 
+constexpr int kMergeGroups = 4;   // most chunk groups of the merge kernel (128 threads each); 1 when chunks are few
+
 template <int HD>
-__global__ void __launch_bounds__(128) decode_merge_kernel(const KernelArgs a, const HeadCfg hc)
+__global__ void __launch_bounds__(kMergeGroups * 128) decode_merge_kernel(const KernelArgs a, const HeadCfg hc)
 {
+    __shared__ float sh_max[kMergeGroups * 4];
+    __shared__ float sh_acc[kMergeGroups][HD];
+    __shared__ float sh_small[kMergeGroups][1 + kMaxSpans];
+
     const int h = blockIdx.x, s = blockIdx.y;
     const int G = a.G, kvh = h / G, gi = h % G;
-    const int L = a.seq_lens[s];
-    const int d = threadIdx.x;
+    const int grp = threadIdx.x >> 7, d = threadIdx.x & 127;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int groups = blockDim.x >> 7, nwarps = blockDim.x >> 5;
     __nv_bfloat16* orow = a.out + ((int64_t)s * a.Hq + h) * HD;
     const int slot = hc.slot[h];
     float* mrow = (slot >= 0 && a.S > 0) ? a.mass + ((int64_t)s * a.P + slot) * a.S : nullptr;
 
+    // the partials are written by the split-K kernel launched just before on the same stream
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    const int L = a.seq_lens[s];
     if (L <= 0 || L > a.max_blocks * kPage) {
         if (threadIdx.x == 0) report(a.status, L <= 0 ? HOOK_ATTN_ERR_INVALID_ARG : HOOK_ATTN_ERR_BOUNDS);
-        if (d < HD) orow[d] = __float2bfloat16(0.f);
-        if (mrow && d < a.S) mrow[d] = 0.f;
+        if (grp == 0 && d < HD) orow[d] = __float2bfloat16(0.f);
+        if (grp == 0 && mrow && d < a.S) mrow[d] = 0.f;
         return;
     }
     const int nchunks = (L + a.chunk - 1) / a.chunk;
@@ -269,24 +280,48 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(const KernelArgs a, c
     const float* part = a.ws + ((((size_t)s * a.Hkv + kvh) * a.max_chunks) * G + gi) * pstride;
     const size_t cstride = (size_t)G * pstride;
 
+    // global maximum of the chunk maxima
     float M = -INFINITY;
-    for (int c = 0; c < nchunks; ++c) M = fmaxf(M, part[c * cstride + HD]);
+    for (int c = threadIdx.x; c < nchunks; c += blockDim.x) M = fmaxf(M, part[c * cstride + HD]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    if (lane == 0) sh_max[warp] = M;
+    __syncthreads();
+    M = sh_max[0];
+    for (int w = 1; w < nwarps; ++w) M = fmaxf(M, sh_max[w]);
+
+    // every group takes the chunks c = grp, grp + 4, ... (several loads in flight per thread); the
+    // groups are then added in group order, so the summation order is fixed from run to run
     float acc = 0.f, lsum = 0.f, macc = 0.f;
-    for (int c = 0; c < nchunks; ++c) {
+#pragma unroll 4
+    for (int c = grp; c < nchunks; c += groups) {
         const float* pc = part + c * cstride;
         const float w = fast_exp2(pc[HD] - M);
         lsum += w * pc[HD + 1];
         if (d < HD) acc += w * pc[d];
         if (mrow && d < a.S) macc += w * pc[HD + 2 + d];
     }
+    if (d < HD) sh_acc[grp][d] = acc;
+    if (d == 0) sh_small[grp][0] = lsum;
+    if (d < a.S) sh_small[grp][1 + d] = macc;
+    __syncthreads();
+    if (grp != 0) return;
+    lsum = sh_small[0][0];
+    for (int g2 = 1; g2 < groups; ++g2) lsum += sh_small[g2][0];
     const float inv = 1.f / lsum;
     if (d < HD) {
-        float val = acc * inv;
+        float val = sh_acc[0][d];
+        for (int g2 = 1; g2 < groups; ++g2) val += sh_acc[g2][d];
+        val *= inv;
         const float al = hc.alpha[h];
         if (al != 0.f) val += al * a.steer[(int64_t)h * HD + d];
         orow[d] = __float2bfloat16(val);
     }
-    if (mrow && d < a.S) mrow[d] = macc * inv;
+    if (mrow && d < a.S) {
+        float mm = sh_small[0][1 + d];
+        for (int g2 = 1; g2 < groups; ++g2) mm += sh_small[g2][1 + d];
+        mrow[d] = mm * inv;
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -297,8 +332,19 @@ static cudaError_t launch_decode_t(const KernelArgs& a, const HeadCfg& hc, cudaS
     decode_splitk_kernel<HD, NS><<<grid, kDecWarps * 32, decode_smem_bytes<HD>(), st>>>(a, hc);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    decode_merge_kernel<HD><<<dim3(a.Hq, a.num_seqs), 128, 0, st>>>(a, hc);
-    return cudaGetLastError();
+    // The merge is launched with programmatic stream serialization: it may be scheduled while the
+    // split-K kernel drains and waits (griddepcontrol.wait) until that kernel's writes are visible.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.Hq, a.num_seqs);
+    cfg.blockDim = dim3((a.max_chunks > 8 ? kMergeGroups : 1) * 128);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_merge_kernel<HD>, a, hc);
 }
 
 template <int HD, int NS>
