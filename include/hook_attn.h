@@ -156,6 +156,42 @@ int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* 
 #define HOOK_ATTN_STATIC_SCRATCH_BYTES (16u << 20)
 int hook_attn_decode_static_scratch(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
 
+/* Analyzer reduction over span masses (Section 2.2: the analyzer turns the re-assembled attention of
+ * the important heads and the configured token ranges into a score, attn_func "sum_normalize";
+ * Section 3: focus score of the instruction, per-passage relevance scores).  The analyzer's body is
+ * not printed in the paper, so the two reductions are this library's reading of its words:
+ *   HOOK_SCORE_MEAN            scores[r][j] = mean over probed heads p of span_mass[r][p][j]
+ *   HOOK_SCORE_SUM_NORMALIZE   scores[r][j] = mean over p of span_mass[r][p][j] / sum_j' span_mass[r][p][j']
+ *                              (a head whose masses sum to zero contributes zero); with the two spans
+ *                              (instruction, data) scores[r][0] is instruction / (instruction + data).
+ * span_mass: device fp32 [rows][num_probed][num_spans] as written by prefill / decode; scores: device
+ * fp32 [rows][num_spans].  Only this small result has to leave the GPU. */
+enum { HOOK_SCORE_MEAN = 0, HOOK_SCORE_SUM_NORMALIZE = 1 };
+int hook_attn_score(hook_attn_handle* handle, const float* span_mass, int32_t rows, int32_t num_probed,
+                    int32_t num_spans, int32_t mode, float* scores, void* cuda_stream);
+
+/* Residual-stream activation steering (Section 1 "Model Steering", Section 3: a steering vector is
+ * injected into a layer of the deployed model): hidden[t][:] += alpha * steer_vec[:] for every token
+ * row t, in place.  hidden: device bf16, num_tokens rows of hidden_size elements, row_stride elements
+ * apart (multiples of 8, 16-byte aligned); steer_vec: device fp32 [hidden_size].  The add is done in
+ * fp32 and rounded once to bf16.  alpha = 0 changes nothing. */
+int hook_steer_residual(hook_attn_handle* handle, void* hidden, const float* steer_vec, float alpha,
+                        int64_t num_tokens, int32_t hidden_size, int64_t row_stride, void* cuda_stream);
+
+/* Raw q/k capture (Section 2.1: the worker's hook keeps, per hooked attention module, the queries of the
+ * last or of all tokens and the keys of all tokens; Section 2.2: the analyzer recomputes attention from
+ * them).  For analyzers that need the raw states rather than span masses.  Reads q, k_cache, block_table,
+ * seq_lens, cu_q_lens (prefill), head_mask (host) and probe_rows of `p`; spans, steering, out and
+ * workspace are ignored.  With P probed heads in ascending order:
+ *   q_out  device bf16 [rows][P][D], rows = total_q (all_tokens) or num_seqs (last_token / decode; a
+ *          sequence without rows in the call gets zeros);               may be NULL
+ *   k_out  device bf16 [sum L_s][P][D]: key t of sequence s at row cu_k_lens[s] + t, taken from the KV
+ *          head of the probed query head;                               may be NULL
+ *   cu_k_lens  device int32 [num_seqs + 1], prefix sums of seq_lens (caller-computed).
+ * Byte-exact copies; block ids are bounds-checked like in the attention calls. */
+int hook_capture_qk(hook_attn_handle* handle, const hook_attn_params* p, int is_decode, void* q_out, void* k_out,
+                    const int32_t* cu_k_lens, void* cuda_stream);
+
 /* Human-readable name of a return / status code. */
 const char* hook_attn_strerror(int code);
 

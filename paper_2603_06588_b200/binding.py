@@ -27,7 +27,9 @@ HOOK_PROBE_ROWS_LAST = 1
 
 EXPORTS = ("hook_attn_create", "hook_attn_destroy", "hook_attn_workspace_bytes",
            "hook_attn_prefill", "hook_attn_decode", "hook_attn_decode_static_scratch",
-           "hook_attn_strerror")
+           "hook_attn_score", "hook_steer_residual", "hook_capture_qk", "hook_attn_strerror")
+HOOK_SCORE_MEAN = 0
+HOOK_SCORE_SUM_NORMALIZE = 1
 STATIC_SCRATCH_BYTES = 16 << 20   # HOOK_ATTN_STATIC_SCRATCH_BYTES
 
 
@@ -80,6 +82,15 @@ def load_library() -> ctypes.CDLL:
             fn = getattr(lib, name)
             fn.restype = ctypes.c_int
             fn.argtypes = [ctypes.c_void_p, ctypes.POINTER(HookAttnParams), ctypes.c_void_p]
+        lib.hook_attn_score.restype = ctypes.c_int
+        lib.hook_attn_score.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                        ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+        lib.hook_steer_residual.restype = ctypes.c_int
+        lib.hook_steer_residual.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float,
+                                            ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p]
+        lib.hook_capture_qk.restype = ctypes.c_int
+        lib.hook_capture_qk.argtypes = [ctypes.c_void_p, ctypes.POINTER(HookAttnParams), ctypes.c_int, ctypes.c_void_p,
+                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         lib.hook_attn_strerror.restype = ctypes.c_char_p
         lib.hook_attn_strerror.argtypes = [ctypes.c_int]
         _lib = lib
@@ -182,6 +193,53 @@ class HookAttn:
             stream = torch.cuda.current_stream(self.device).cuda_stream
         return int(self._lib.hook_attn_decode_static_scratch(self._h, ctypes.byref(params),
                                                              ctypes.c_void_p(stream)))
+
+    def _stream(self, stream):
+        return ctypes.c_void_p(torch.cuda.current_stream(self.device).cuda_stream if stream is None else stream)
+
+    def hook_attn_score(self, span_mass: torch.Tensor, mode: int = HOOK_SCORE_SUM_NORMALIZE, scores=None, stream=None):
+        """Analyzer reduction: ``span_mass`` fp32 ``[R, P, S]`` (device) -> ``scores`` fp32 ``[R, S]``."""
+        rows, nprobed, nspans = span_mass.shape
+        assert span_mass.dtype == torch.float32 and span_mass.is_contiguous()
+        if scores is None:
+            scores = torch.empty((rows, nspans), dtype=torch.float32, device=span_mass.device)
+        rc = int(self._lib.hook_attn_score(self._h, span_mass.data_ptr(), rows, nprobed, nspans, int(mode),
+                                           scores.data_ptr(), self._stream(stream)))
+        if rc != HOOK_ATTN_OK:
+            raise HookAttnError(rc, "hook_attn_score")
+        return scores
+
+    def hook_steer_residual(self, hidden: torch.Tensor, steer_vec: torch.Tensor, alpha: float, stream=None):
+        """Residual-stream steering in place: ``hidden`` bf16 ``[T, H]`` (device, rows may be strided),
+        ``steer_vec`` fp32 ``[H]``."""
+        assert hidden.dtype == torch.bfloat16 and hidden.dim() == 2 and hidden.stride(1) == 1
+        assert steer_vec.dtype == torch.float32 and steer_vec.is_contiguous()
+        rc = int(self._lib.hook_steer_residual(self._h, hidden.data_ptr(), steer_vec.data_ptr(), float(alpha),
+                                               hidden.shape[0], hidden.shape[1], hidden.stride(0), self._stream(stream)))
+        if rc != HOOK_ATTN_OK:
+            raise HookAttnError(rc, "hook_steer_residual")
+        return hidden
+
+    def hook_capture_qk(self, is_decode: bool, *, q, k_cache, v_cache, block_table, seq_lens, cu_q_lens=None,
+                        head_mask=None, probe_rows=HOOK_PROBE_ROWS_ALL, status=None, stream=None, **_ignored):
+        """Raw q/k capture of the probed heads.  Returns ``(q_out [rows, P, D], k_out [sum L, P, D], cu_k_lens)``."""
+        nprobed = 0 if head_mask is None else int((head_mask != 0).sum())
+        total_q, hq, d = q.shape
+        last_only = is_decode or probe_rows == HOOK_PROBE_ROWS_LAST
+        rows = int(seq_lens.shape[0]) if last_only else int(total_q)
+        cu_k = torch.zeros(seq_lens.shape[0] + 1, dtype=torch.int32, device=q.device)
+        cu_k[1:] = torch.cumsum(seq_lens, 0)
+        total_k = int(cu_k[-1].item())
+        q_out = torch.zeros((rows, nprobed, d), dtype=torch.bfloat16, device=q.device)
+        k_out = torch.zeros((total_k, nprobed, d), dtype=torch.bfloat16, device=q.device)
+        p, keep = make_params(q=q, k_cache=k_cache, v_cache=v_cache, block_table=block_table, seq_lens=seq_lens,
+                              cu_q_lens=cu_q_lens, head_mask=head_mask, probe_rows=probe_rows, status=status)
+        rc = int(self._lib.hook_capture_qk(self._h, ctypes.byref(p), int(bool(is_decode)), q_out.data_ptr(),
+                                           k_out.data_ptr(), cu_k.data_ptr(), self._stream(stream)))
+        del keep
+        if rc != HOOK_ATTN_OK:
+            raise HookAttnError(rc, "hook_capture_qk")
+        return q_out, k_out, cu_k
 
     # -- convenience ---------------------------------------------------------------------
     def plan(self, is_decode: bool, *, q, k_cache, v_cache, block_table, seq_lens, cu_q_lens=None,

@@ -21,6 +21,12 @@ int prefill_mma_tiles_upper_bound(int total_q, int num_seqs);
 cudaError_t configure_prefill_tc();
 bool prefill_tc_supported(const KernelArgs& a, int head_dim);
 cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, cudaStream_t st);
+// extras.cu
+cudaError_t launch_score(const float* mass, float* scores, int rows, int P, int S, int mode, cudaStream_t st);
+cudaError_t launch_steer_residual(__nv_bfloat16* hidden, const float* vec, float alpha, int64_t tokens, int hidden_size,
+                                  int64_t row_stride, int num_sms, cudaStream_t st);
+cudaError_t launch_capture(const KernelArgs& a, const HeadCfg& hc, int head_dim, bool decode, __nv_bfloat16* q_out,
+                           __nv_bfloat16* k_out, const int32_t* cu_k, cudaStream_t st);
 }  // namespace hook_attn
 
 using namespace hook_attn;
@@ -252,6 +258,60 @@ int hook_attn_decode_static_scratch(hook_attn_handle* handle, const hook_attn_pa
     a.ws = scratch;   // every partial the merge reads is written by the split-K kernel of the same call:
                       // nothing in the array has to start at zero, stale contents are never read
     cudaError_t e = launch_decode(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
+}
+
+int hook_attn_score(hook_attn_handle* handle, const float* span_mass, int32_t rows, int32_t num_probed, int32_t num_spans,
+                    int32_t mode, float* scores, void* cuda_stream)
+{
+    if (rows < 0 || num_probed <= 0 || num_spans <= 0) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (mode != HOOK_SCORE_MEAN && mode != HOOK_SCORE_SUM_NORMALIZE) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (num_spans > kMaxSpans) return HOOK_ATTN_ERR_UNSUPPORTED;
+    if (rows > 0 && (!span_mass || !scores)) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (rows == 0) return HOOK_ATTN_OK;
+    cudaError_t e = launch_score(span_mass, scores, rows, num_probed, num_spans, mode, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
+}
+
+int hook_steer_residual(hook_attn_handle* handle, void* hidden, const float* steer_vec, float alpha, int64_t num_tokens,
+                        int32_t hidden_size, int64_t row_stride, void* cuda_stream)
+{
+    if (num_tokens < 0 || hidden_size <= 0 || row_stride < hidden_size || !isfinite(alpha)) return HOOK_ATTN_ERR_INVALID_ARG;
+    if ((hidden_size & 7) || (row_stride & 7)) return HOOK_ATTN_ERR_UNSUPPORTED;
+    if (num_tokens > 0 && (!hidden || !steer_vec)) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(steer_vec)) return HOOK_ATTN_ERR_UNSUPPORTED;
+    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (num_tokens == 0 || alpha == 0.0f) return HOOK_ATTN_OK;   // alpha = 0 leaves every bit in place
+    cudaError_t e = launch_steer_residual(static_cast<__nv_bfloat16*>(hidden), steer_vec, alpha, num_tokens, hidden_size,
+                                          row_stride, handle->num_sms, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
+}
+
+int hook_capture_qk(hook_attn_handle* handle, const hook_attn_params* p, int is_decode, void* q_out, void* k_out,
+                    const int32_t* cu_k_lens, void* cuda_stream)
+{
+    KernelArgs a;
+    HeadCfg hc;
+    hook_attn_params q = {};
+    if (p) {
+        q = *p;
+        q.out = const_cast<void*>(p->q);   // the capture writes no attention output; keep the shared checks satisfied
+        q.num_spans = 0;                   // spans play no role here
+    }
+    int rc = prepare(p ? &q : nullptr, is_decode != 0, a, hc);
+    if (rc != HOOK_ATTN_OK) return rc;
+    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (p->num_seqs == 0 || p->total_q == 0) return HOOK_ATTN_OK;
+    int probed = 0;
+    for (int h = 0; h < p->num_q_heads; ++h)
+        if (p->head_mask && p->head_mask[h]) hc.slot[h] = (int8_t)probed++; else hc.slot[h] = -1;
+    if (probed == 0) return HOOK_ATTN_OK;   // nothing is hooked
+    a.P = probed;
+    if (k_out && !cu_k_lens) return HOOK_ATTN_ERR_INVALID_ARG;
+    if ((q_out && !aligned16(q_out)) || (k_out && !aligned16(k_out))) return HOOK_ATTN_ERR_UNSUPPORTED;
+    cudaError_t e = launch_capture(a, hc, p->head_dim, is_decode != 0, static_cast<__nv_bfloat16*>(q_out),
+                                   static_cast<__nv_bfloat16*>(k_out), cu_k_lens, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
 }
 

@@ -271,7 +271,9 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
     }
     const int nmax = max(ntiles[0], ntiles[1]);
     const int slot = (NS > 0) ? hc.slot[h] : -1;
-    const bool probe = (NS > 0) && slot >= 0;
+    // in last-token mode only the pair of tiles that holds the sequence's last row carries the probe
+    const bool probe = (NS > 0) && slot >= 0 &&
+                       (a.probe_rows == HOOK_PROBE_ROWS_ALL || (n - 1 >= row0[0] && n - 1 < row0[0] + 2 * kBM));
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t sQ[2] = {smem_base, smem_base + kTileBytes};
