@@ -48,6 +48,13 @@ WORKLOADS = {
 }
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu captures
+# summarised under profiles/ (None where no capture of the current kernel exists).
+DRAM_TRAFFIC = {
+    "cfg2_decode": 625.09e6 + 6.44e6,     # profiles/decode_splitk_kernel__cfg2_decode.md
+}
+
+
 def make_workload(name: str):
     if name == "cfg2_decode":
         return inputs.config2_decode()
@@ -176,23 +183,25 @@ def oracle_sample(case, budget_s: float):
     the number of tokens the timing is scaled to (rows evaluated, weighted by visible keys so that
     the figure stays a tokens/s of the same workload)."""
     total_pairs = case.visible_pairs()
-    # the oracle sustains roughly 3e8 (key, d) multiply-adds per core-second; size by that
+    # the oracle sustains very roughly 5e8 (key, d) multiply-adds per core-second over K and V
     macs_per_row_key = 2 * case.head_dim * case.num_q_heads
-    budget_pairs = budget_s * 2.5e9 / macs_per_row_key
+    budget_pairs = budget_s * 5e8 * max(1, os.cpu_count() or 1) / macs_per_row_key
     if total_pairs <= budget_pairs:
-        return None if False else list(range(case.total_q)), f"all {case.total_q} query rows x {case.num_q_heads} heads", case.total_q
-    rows = inputs.sample_rows(case, extra_random=0)
+        return list(range(case.total_q)), f"all {case.total_q} query rows x {case.num_q_heads} heads", case.total_q
+    rows = inputs.sample_rows(case, extra_random=256)
     cu = case.cu_q_lens.tolist()
     Ls = case.seq_lens.tolist()
+    order = torch.randperm(len(rows), generator=torch.Generator().manual_seed(11)).tolist()
     picked, pairs = [], 0
-    stride = max(1, len(rows) // 64)
-    for r in rows[::stride]:
-        s = max(i for i in range(case.num_seqs) if cu[i] <= r)
+    for idx in order:
+        r = rows[idx]
+        s = max(i for i in range(case.num_seqs) if cu[i] <= r and cu[i + 1] > cu[i])
         pos = Ls[s] - (cu[s + 1] - cu[s]) + (r - cu[s])
         if pairs + pos + 1 > budget_pairs and picked:
             break
         picked.append(r)
         pairs += pos + 1
+    picked.sort()
     tokens = case.total_q * pairs / total_pairs
     return picked, (f"{len(picked)} sampled query rows x {case.num_q_heads} heads ({pairs} of {total_pairs} visible pairs per head); "
                     "tokens/s extrapolated by visible-pair count"), tokens
@@ -337,10 +346,8 @@ def main():
     t_e2e = ev0.elapsed_time(ev1) / 1e3 / n_e2e
     clocks_all = sampler2.stop()
 
-    if dist:
-        t = torch.tensor([t_hook, t_e2e], dtype=torch.float64, device=f"cuda:{local}")
-        td.all_reduce(t, op=td.ReduceOp.MAX)
-        t_hook, t_e2e = float(t[0]), float(t[1])
+    from paper_2603_06588_b200 import replicas
+    t_hook, t_e2e = replicas.max_over_ranks([t_hook, t_e2e], torch.device("cuda", local))
 
     if rank == 0:
         peaks = load_peaks()
@@ -355,7 +362,7 @@ def main():
             peak, unit = (peaks["bf16_tflops"] if t_hook < 2.0 else peaks["bf16_tflops_sustained"]), "TFLOP/s"
         clocks = clocks_timed if clocks_timed["samples"] >= 3 else clocks_all
         line = {
-            "metric": METRIC, "value": world * tokens / per_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": METRIC, "value": replicas.replica_throughput(tokens, per_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}",
@@ -363,14 +370,14 @@ def main():
                        else "L2 flushed between iterations (256 MB write)",
                        "replicas": world, "kv_cache": "resident in HBM (state, not a per-step input)"},
             "roofline": {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                         "traffic": None, "peak_source": f"of {peaks['source']}",
+                         "traffic": DRAM_TRAFFIC.get(args.workload), "peak_source": f"of {peaks['source']}",
                          "kernel": "decode_splitk_kernel (+ decode_merge_kernel; duration = whole step, conservative)"
-                         if case.is_decode else "prefill kernel (one launch per step)",
+                         if case.is_decode else "prefill_tc_kernel (one launch per step)",
                          "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
                          "frac_of_datasheet": achieved / (8000.0 if bound == "hbm" else 2250.0)},
             "hook_overhead": overhead,
             "ms_per_step_hooks_off": statistics.median(tp) * 1e3,
-            "e2e": {"value": world * tokens / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "e2e": {"value": replicas.replica_throughput(tokens, t_e2e, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": t_e2e * 1e3},
             "gpu_launches": launches_per_step * args.steps,
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
