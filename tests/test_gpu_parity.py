@@ -287,3 +287,37 @@ def test_strided_cache_views(eng):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert torch.equal(out.view(torch.int16), out_ref.view(torch.int16)) and torch.equal(mass, mass_ref)
+
+
+def test_calls_are_capturable_in_a_cuda_graph(eng):
+    """A launch-bound layer loop (several prefill and decode calls) captured once and replayed gives
+    the same bits as the eager calls: the entry points neither synchronise nor allocate."""
+    pf = [inputs.config3_prefill(layer=l, num_seqs=1, tokens=384, force_probe=True) for l in range(3)]
+    dec = inputs.config2_decode(num_seqs=8, lo=100, hi=1500)
+    plans, eager = [], []
+    for case in pf + [dec]:
+        kw = binding.case_to_device(case)
+        plan = eng.plan(case.is_decode, **kw)
+        plan.run()
+        plans.append(plan)
+    torch.cuda.synchronize()
+    eager = [(p.out.clone(), None if p.span_mass is None else p.span_mass.clone()) for p in plans]
+    for p in plans:
+        p.out.zero_()
+        if p.span_mass is not None:
+            p.span_mass.zero_()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for p in plans:
+                p.run()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    for p, (o, m) in zip(plans, eager):
+        assert torch.equal(p.out.view(torch.int16), o.view(torch.int16))
+        if m is not None:
+            assert torch.equal(p.span_mass, m)
