@@ -247,20 +247,23 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_splitk_kernel(const Ker
     }
 }
 
-constexpr int kMergeGroups = 4;   // most chunk groups of the merge kernel (128 threads each); 1 when chunks are few
+constexpr int kMergeMaxWarps = 16;   // warps of the merge kernel when a sequence has many chunks (4 otherwise)
 
+// One CTA per (query head, sequence).  Warp w folds the chunks w, w + nwarps, ... with an online
+// rescale (all loads of a chunk are independent of the previous chunk's arithmetic, so several
+// chunks are in flight); the warps are then combined in warp order by the first 128 threads.  The
+// order of every floating-point sum is fixed by (chunk, warp) indices only: run-to-run bit-identical.
 template <int HD>
-__global__ void __launch_bounds__(kMergeGroups * 128) decode_merge_kernel(const KernelArgs a, const HeadCfg hc)
+__global__ void __launch_bounds__(kMergeMaxWarps * 32) decode_merge_kernel(const KernelArgs a, const HeadCfg hc)
 {
-    __shared__ float sh_max[kMergeGroups * 4];
-    __shared__ float sh_acc[kMergeGroups][HD];
-    __shared__ float sh_small[kMergeGroups][1 + kMaxSpans];
+    constexpr int EPL = HD / 32;                       // output elements per lane
+    __shared__ float sh_acc[kMergeMaxWarps][HD];
+    __shared__ float sh_small[kMergeMaxWarps][2 + kMaxSpans];   // M, l, s[0..7]
 
     const int h = blockIdx.x, s = blockIdx.y;
     const int G = a.G, kvh = h / G, gi = h % G;
-    const int grp = threadIdx.x >> 7, d = threadIdx.x & 127;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int groups = blockDim.x >> 7, nwarps = blockDim.x >> 5;
+    const int nwarps = blockDim.x >> 5;
     __nv_bfloat16* orow = a.out + ((int64_t)s * a.Hq + h) * HD;
     const int slot = hc.slot[h];
     float* mrow = (slot >= 0 && a.S > 0) ? a.mass + ((int64_t)s * a.P + slot) * a.S : nullptr;
@@ -271,57 +274,61 @@ __global__ void __launch_bounds__(kMergeGroups * 128) decode_merge_kernel(const 
     const int L = a.seq_lens[s];
     if (L <= 0 || L > a.max_blocks * kPage) {
         if (threadIdx.x == 0) report(a.status, L <= 0 ? HOOK_ATTN_ERR_INVALID_ARG : HOOK_ATTN_ERR_BOUNDS);
-        if (grp == 0 && d < HD) orow[d] = __float2bfloat16(0.f);
-        if (grp == 0 && mrow && d < a.S) mrow[d] = 0.f;
+        if ((int)threadIdx.x < HD) orow[threadIdx.x] = __float2bfloat16(0.f);
+        if (mrow && (int)threadIdx.x < a.S) mrow[threadIdx.x] = 0.f;
         return;
     }
     const int nchunks = (L + a.chunk - 1) / a.chunk;
     const size_t pstride = decode_partial_stride(HD);
     const float* part = a.ws + ((((size_t)s * a.Hkv + kvh) * a.max_chunks) * G + gi) * pstride;
     const size_t cstride = (size_t)G * pstride;
+    const bool want_mass = mrow != nullptr;
 
-    // global maximum of the chunk maxima
-    float M = -INFINITY;
-    for (int c = threadIdx.x; c < nchunks; c += blockDim.x) M = fmaxf(M, part[c * cstride + HD]);
+    float M = -INFINITY, lsum = 0.f, sacc = 0.f, acc[EPL];
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    if (lane == 0) sh_max[warp] = M;
-    __syncthreads();
-    M = sh_max[0];
-    for (int w = 1; w < nwarps; ++w) M = fmaxf(M, sh_max[w]);
-
-    // every group takes the chunks c = grp, grp + 4, ... (several loads in flight per thread); the
-    // groups are then added in group order, so the summation order is fixed from run to run
-    float acc = 0.f, lsum = 0.f, macc = 0.f;
+    for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
 #pragma unroll 4
-    for (int c = grp; c < nchunks; c += groups) {
+    for (int c = warp; c < nchunks; c += nwarps) {
         const float* pc = part + c * cstride;
-        const float w = fast_exp2(pc[HD] - M);
-        lsum += w * pc[HD + 1];
-        if (d < HD) acc += w * pc[d];
-        if (mrow && d < a.S) macc += w * pc[HD + 2 + d];
+        const float mc = pc[HD], lc = pc[HD + 1];
+        float oc[EPL];
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) oc[e] = pc[lane + 32 * e];
+        const float sc = (want_mass && lane < a.S) ? pc[HD + 2 + lane] : 0.f;
+        const float Mn = fmaxf(M, mc);
+        const float fo = fast_exp2(M - Mn), fc = fast_exp2(mc - Mn);   // M = -inf on the first chunk: fo = 0
+        M = Mn;
+        lsum = lsum * fo + lc * fc;
+        sacc = sacc * fo + sc * fc;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] = acc[e] * fo + oc[e] * fc;
     }
-    if (d < HD) sh_acc[grp][d] = acc;
-    if (d == 0) sh_small[grp][0] = lsum;
-    if (d < a.S) sh_small[grp][1 + d] = macc;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) sh_acc[warp][lane + 32 * e] = acc[e];
+    if (lane == 0) { sh_small[warp][0] = M; sh_small[warp][1] = lsum; }
+    if (lane < kMaxSpans) sh_small[warp][2 + lane] = sacc;
     __syncthreads();
-    if (grp != 0) return;
-    lsum = sh_small[0][0];
-    for (int g2 = 1; g2 < groups; ++g2) lsum += sh_small[g2][0];
-    const float inv = 1.f / lsum;
+
+    const int d = threadIdx.x;
+    if (d >= 128) return;
+    const int used = min(nwarps, nchunks);             // warps that folded at least one chunk
+    float Mg = sh_small[0][0];
+    for (int w = 1; w < used; ++w) Mg = fmaxf(Mg, sh_small[w][0]);
+    float ltot = 0.f, val = 0.f, mm = 0.f;
+    for (int w = 0; w < used; ++w) {
+        const float f = fast_exp2(sh_small[w][0] - Mg);
+        ltot += f * sh_small[w][1];
+        if (d < HD) val += f * sh_acc[w][d];
+        if (d < kMaxSpans) mm += f * sh_small[w][2 + d];
+    }
+    const float inv = 1.f / ltot;
     if (d < HD) {
-        float val = sh_acc[0][d];
-        for (int g2 = 1; g2 < groups; ++g2) val += sh_acc[g2][d];
         val *= inv;
         const float al = hc.alpha[h];
         if (al != 0.f) val += al * a.steer[(int64_t)h * HD + d];
         orow[d] = __float2bfloat16(val);
     }
-    if (mrow && d < a.S) {
-        float mm = sh_small[0][1 + d];
-        for (int g2 = 1; g2 < groups; ++g2) mm += sh_small[g2][1 + d];
-        mrow[d] = mm * inv;
-    }
+    if (mrow && d < a.S) mrow[d] = mm * inv;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -336,7 +343,7 @@ static cudaError_t launch_decode_t(const KernelArgs& a, const HeadCfg& hc, cudaS
     // split-K kernel drains and waits (griddepcontrol.wait) until that kernel's writes are visible.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.Hq, a.num_seqs);
-    cfg.blockDim = dim3((a.max_chunks > 8 ? kMergeGroups : 1) * 128);
+    cfg.blockDim = dim3((a.max_chunks > 8 ? kMergeMaxWarps : 4) * 32);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
