@@ -192,6 +192,14 @@ int hook_steer_residual(hook_attn_handle* handle, void* hidden, const float* ste
 int hook_capture_qk(hook_attn_handle* handle, const hook_attn_params* p, int is_decode, void* q_out, void* k_out,
                     const int32_t* cu_k_lens, void* cuda_stream);
 
+/* Self-test of the kernels' bounded waits (the paper has no counterpart; it backs the failure
+ * behaviour stated above).  Launches one small kernel that waits on a barrier nothing ever signals.
+ * After `limit_ns` (1 .. 1e9) the wait gives up, the kernel writes HOOK_ATTN_ERR_TIMEOUT into the
+ * device word `status` (zeroed by the caller), stores the time it waited into the optional device
+ * word `waited_ns`, and returns normally: no trap, no hang, the context stays usable. */
+int hook_attn_selftest_wait_limit(hook_attn_handle* handle, int32_t* status, uint64_t limit_ns, uint64_t* waited_ns,
+                                  void* cuda_stream);
+
 /* Human-readable name of a return / status code. */
 const char* hook_attn_strerror(int code);
 

@@ -27,7 +27,8 @@ HOOK_PROBE_ROWS_LAST = 1
 
 EXPORTS = ("hook_attn_create", "hook_attn_destroy", "hook_attn_workspace_bytes",
            "hook_attn_prefill", "hook_attn_decode", "hook_attn_decode_static_scratch",
-           "hook_attn_score", "hook_steer_residual", "hook_capture_qk", "hook_attn_strerror")
+           "hook_attn_score", "hook_steer_residual", "hook_capture_qk", "hook_attn_selftest_wait_limit",
+           "hook_attn_strerror")
 HOOK_SCORE_MEAN = 0
 HOOK_SCORE_SUM_NORMALIZE = 1
 STATIC_SCRATCH_BYTES = 16 << 20   # HOOK_ATTN_STATIC_SCRATCH_BYTES
@@ -91,6 +92,9 @@ def load_library() -> ctypes.CDLL:
         lib.hook_capture_qk.restype = ctypes.c_int
         lib.hook_capture_qk.argtypes = [ctypes.c_void_p, ctypes.POINTER(HookAttnParams), ctypes.c_int, ctypes.c_void_p,
                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        lib.hook_attn_selftest_wait_limit.restype = ctypes.c_int
+        lib.hook_attn_selftest_wait_limit.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p,
+                                                      ctypes.c_void_p]
         lib.hook_attn_strerror.restype = ctypes.c_char_p
         lib.hook_attn_strerror.argtypes = [ctypes.c_int]
         _lib = lib
@@ -193,6 +197,17 @@ class HookAttn:
             stream = torch.cuda.current_stream(self.device).cuda_stream
         return int(self._lib.hook_attn_decode_static_scratch(self._h, ctypes.byref(params),
                                                              ctypes.c_void_p(stream)))
+
+    def selftest_wait_limit(self, limit_ns: int = 200_000_000, stream=None):
+        """Run the bounded-wait self-test; returns ``(status_code, waited_ns)`` read back from the device."""
+        status = torch.zeros(1, dtype=torch.int32, device=self.device)
+        waited = torch.zeros(1, dtype=torch.int64, device=self.device)
+        rc = int(self._lib.hook_attn_selftest_wait_limit(self._h, status.data_ptr(), int(limit_ns), waited.data_ptr(),
+                                                         self._stream(stream)))
+        if rc != HOOK_ATTN_OK:
+            raise HookAttnError(rc, "hook_attn_selftest_wait_limit")
+        torch.cuda.synchronize(self.device)
+        return int(status.item()), int(waited.item())
 
     def _stream(self, stream):
         return ctypes.c_void_p(torch.cuda.current_stream(self.device).cuda_stream if stream is None else stream)

@@ -21,6 +21,7 @@ int prefill_mma_tiles_upper_bound(int total_q, int num_seqs);
 cudaError_t configure_prefill_tc();
 bool prefill_tc_supported(const KernelArgs& a, int head_dim);
 cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, cudaStream_t st);
+cudaError_t launch_wait_selftest(int32_t* status, uint64_t limit_ns, uint64_t* waited_ns, cudaStream_t st);
 // extras.cu
 cudaError_t launch_score(const float* mass, float* scores, int rows, int P, int S, int mode, cudaStream_t st);
 cudaError_t launch_steer_residual(__nv_bfloat16* hidden, const float* vec, float alpha, int64_t tokens, int hidden_size,
@@ -312,6 +313,15 @@ int hook_capture_qk(hook_attn_handle* handle, const hook_attn_params* p, int is_
     if ((q_out && !aligned16(q_out)) || (k_out && !aligned16(k_out))) return HOOK_ATTN_ERR_UNSUPPORTED;
     cudaError_t e = launch_capture(a, hc, p->head_dim, is_decode != 0, static_cast<__nv_bfloat16*>(q_out),
                                    static_cast<__nv_bfloat16*>(k_out), cu_k_lens, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
+}
+
+int hook_attn_selftest_wait_limit(hook_attn_handle* handle, int32_t* status, uint64_t limit_ns, uint64_t* waited_ns,
+                                  void* cuda_stream)
+{
+    if (!status || limit_ns == 0 || limit_ns > 1000000000ull) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    cudaError_t e = launch_wait_selftest(status, limit_ns, waited_ns, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
 }
 

@@ -90,14 +90,14 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after about two seconds.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+// Bounded wait: gives up after `limit_ns` (two seconds unless stated otherwise).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns = 2000000000ull)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u && global_timer_ns() - t0 > 2000000000ull) return false;
+        if ((it & 255u) == 255u && global_timer_ns() - t0 > limit_ns) return false;
     }
 }
 
@@ -688,6 +688,31 @@ cudaError_t configure_one()
 }
 
 }  // namespace
+
+// Self-test of the bounded waits: one CTA waits on an mbarrier that nothing ever arrives at.  The
+// wait must run out after `limit_ns`, the kernel must report HOOK_ATTN_ERR_TIMEOUT through the status
+// word and return normally, leaving the context usable.
+__global__ void wait_selftest_kernel(int32_t* status, uint64_t limit_ns, uint64_t* waited_ns)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const uint64_t t0 = global_timer_ns();
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar), 0, limit_ns));
+    if (threadIdx.x == 0) {
+        if (!ok) report(status, HOOK_ATTN_ERR_TIMEOUT);
+        if (waited_ns) *waited_ns = global_timer_ns() - t0;
+    }
+}
+
+cudaError_t launch_wait_selftest(int32_t* status, uint64_t limit_ns, uint64_t* waited_ns, cudaStream_t st)
+{
+    wait_selftest_kernel<<<1, 32, 0, st>>>(status, limit_ns, waited_ns);
+    return cudaGetLastError();
+}
 
 cudaError_t configure_prefill_tc()
 {

@@ -321,3 +321,13 @@ def test_calls_are_capturable_in_a_cuda_graph(eng):
         assert torch.equal(p.out.view(torch.int16), o.view(torch.int16))
         if m is not None:
             assert torch.equal(p.span_mass, m)
+
+
+def test_a_wait_that_nothing_ends_runs_out_and_reports_a_timeout(eng):
+    """Failure detection without a fault: a kernel waits on a barrier that is never signalled; the
+    bounded wait gives up after its limit, the status word carries the timeout code, the kernel
+    returns normally and the context keeps working."""
+    st, waited = eng.selftest_wait_limit(limit_ns=100_000_000)
+    assert st == binding.HOOK_ATTN_ERR_TIMEOUT
+    assert 100_000_000 <= waited < 1_000_000_000
+    check(eng, inputs.config2_decode(num_seqs=4, lo=50, hi=300))     # the context is still usable
