@@ -118,7 +118,7 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "sm_mhz_min": None, "power_w": None}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -128,7 +128,7 @@ class ClockSampler:
             self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         for line in self.file.read().splitlines():
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
@@ -136,6 +136,7 @@ class ClockSampler:
             try:
                 sm.append(float(f[1]))
                 mx.append(float(f[2]))
+                pw.append(float(f[3]))
             except ValueError:
                 continue
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
@@ -145,7 +146,8 @@ class ClockSampler:
         os.unlink(self.file.name)
         if sm:
             # samples under load: the upper half of the observed clocks (idle samples sit low)
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm),
+                       sm_mhz_min=min(sm), power_w=statistics.median(pw) if pw else None)
         return out
 
 
@@ -480,7 +482,7 @@ def main():
                     "ms_per_step": t_e2e * 1e3},
             "gpu_launches": launches_per_step * args.steps,
             "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                       "samples": clocks["samples"]},
+                       "samples": clocks["samples"], "sm_mhz_min": clocks["sm_mhz_min"], "power_w": clocks["power_w"]},
         }
         if not args.no_cpu_baseline:
             from oracle import oracle
