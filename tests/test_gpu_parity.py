@@ -331,3 +331,18 @@ def test_a_wait_that_nothing_ends_runs_out_and_reports_a_timeout(eng):
     assert st == binding.HOOK_ATTN_ERR_TIMEOUT
     assert 100_000_000 <= waited < 1_000_000_000
     check(eng, inputs.config2_decode(num_seqs=4, lo=50, hi=300))     # the context is still usable
+
+
+def test_chunk_on_a_very_long_context(eng):
+    """A 128-row chunk appended to a context of more than 131072 keys: the key-tile loop runs past the
+    precomputed span table of the prefill kernel, block tables are thousands of pages long, and the
+    spans sit on both sides of that boundary."""
+    L, n = 140_003, 128
+    spans = torch.tensor([[[0, 70_000], [70_000, 131_100], [131_100, 139_950], [139_950, L]]], dtype=torch.int32)
+    case = inputs.make_case("long_chunk", is_decode=False, seq_lens=[L], q_lens=[n], num_q_heads=2, num_kv_heads=1,
+                            head_dim=128, seed=31, spans=spans, head_mask=torch.tensor([1, 1], dtype=torch.uint8),
+                            alpha=torch.tensor([0.0, 1.5]), steer=True, pool=1.0)
+    check(eng, case, rows=[0, 1, 52, 53, 54, 126, 127])
+    dec = inputs.replace(case, is_decode=True, q=case.q[-1:].contiguous(), cu_q_lens=torch.tensor([0, 1], dtype=torch.int32),
+                         probe_rows=inputs.PROBE_ROWS_LAST)
+    check(eng, dec)
