@@ -404,13 +404,15 @@ def main():
     # hook overhead: same kernels with hooks disabled, interleaved with hooked passes
     sampler2 = ClockSampler(local)
     sampler2.start()
-    reps = 5
-    n_ov = max(10, args.steps // reps)
+    reps = 7
+    n_ov = max(20, min(args.steps, 200))
     th, tp = [], []
     for _ in range(reps):
         tp.append(run_timed(n_ov, plain) / n_ov)
         th.append(run_timed(n_ov, hooked) / n_ov)
-    overhead = statistics.median(th) / statistics.median(tp) - 1.0
+    # median of the ratios of neighbouring (hooked, plain) passes: clock drift under the power cap
+    # moves both members of a pair alike
+    overhead = statistics.median(h / p for h, p in zip(th, tp)) - 1.0
 
     # end to end through the public call with host buffers: the step's inputs (queries, tables,
     # lengths, spans) come from pinned host memory and the results go back to the host every step;
