@@ -346,3 +346,12 @@ def test_chunk_on_a_very_long_context(eng):
     dec = inputs.replace(case, is_decode=True, q=case.q[-1:].contiguous(), cu_q_lens=torch.tensor([0, 1], dtype=torch.int32),
                          probe_rows=inputs.PROBE_ROWS_LAST)
     check(eng, dec)
+
+
+def test_small_head_dim_128_calls_take_the_warp_mma_kernel(eng):
+    """Fewer than 128 query rows at head_dim 128 are served by the warp-level MMA kernel."""
+    case = inputs.make_case("tiny128", is_decode=False, seq_lens=[90, 33], q_lens=[40, 33], num_q_heads=6, num_kv_heads=2,
+                            head_dim=128, seed=17, num_spans=3, head_mask=torch.tensor([1, 0, 1, 0, 0, 1], dtype=torch.uint8),
+                            alpha=torch.tensor([0.0, 0.5, 0.0, 0.0, -1.0, 0.0]), steer=True, poison=True)
+    assert case.total_q < 128
+    check(eng, case)
