@@ -52,7 +52,8 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu captures
 # summarised under profiles/ (None where no capture of the current kernel exists).
 DRAM_TRAFFIC = {
-    "cfg2_decode": 625.09e6 + 6.44e6,     # profiles/decode_splitk_kernel__cfg2_decode.md
+    "cfg2_decode": 625.15e6 + 6.59e6,     # profiles/decode_splitk_kernel__cfg2_decode.md
+    "cfg3_prefill_small": 50.41e6 + 3.83e6,   # profiles/prefill_tc_kernel__cfg3_prefill_small.md
 }
 
 
