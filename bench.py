@@ -44,6 +44,8 @@ WORKLOADS = {
     "cfg4_decode": "mixed batch, decode part: 256 seqs, ctx U[1024,8192], Hq28/Hkv4, D128, 14 probed heads, 4 spans, 8 steered heads",
     "cfg4_prefill": "mixed batch, prefill part: 2 chunks of 2048 tokens on 4096-token contexts, Hq28/Hkv4, D128",
     "cfg4_mixed": "mixed chunked batch: the 256-sequence decode call and the 2-chunk prefill call of one step, issued on two streams",
+    "steer_residual": "residual-stream steering: hidden[32768 x 4096] bf16 += alpha * vec, in place",
+    "capture_qk": "raw q/k capture of the 16 probed heads of the decode batch (64 seqs, ctx U[512,4096])",
     "cfg5_decode": "long context decode: 4 seqs at 32768+ keys, Hq64/Hkv8, D128, 64 probed heads, 8 spans, 8 steered heads",
     "cfg5_prefill": "long context prefill: 4 seqs x 32768 tokens causal, Hq64/Hkv8, D128, 64 probed heads, 8 spans, 8 steered heads",
 }
@@ -212,6 +214,80 @@ def oracle_sample(case, budget_s: float):
 
 
 # ------------------------------------------------------------------------------------------------
+def run_extra(args):
+    """The two HBM-bound companions of the attention path: residual steering and raw q/k capture."""
+    from paper_2603_06588_b200 import binding
+    args.warmup = max(args.warmup, 3)
+    torch.cuda.set_device(0)
+    eng = binding.HookAttn(0)
+    g = torch.Generator().manual_seed(inputs.BASE_SEED + 77)
+    if args.workload == "steer_residual":
+        T, H = 32768, 4096
+        hidden = torch.randn(T, H, generator=g).to(torch.bfloat16).cuda()
+        vec = torch.randn(H, generator=g).cuda()
+        step = lambda: eng.hook_steer_residual(hidden, vec, 1e-3)
+        alg_bytes, tokens, launches, kernel = 2 * T * H * 2 + H * 4, T, 1, "steer_residual_kernel"
+        host_in, host_out = hidden.cpu().pin_memory(), torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
+
+        def e2e():
+            hidden.copy_(host_in, non_blocking=True)
+            step()
+            host_out.copy_(hidden, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+        h2d = d2h = T * H * 2
+    else:
+        case = inputs.config2_decode()
+        kw = binding.case_to_device(case)
+        q_out, k_out, cu_k = eng.hook_capture_qk(True, **kw)
+        step = lambda: eng.hook_capture_qk(True, q_out=q_out, k_out=k_out, cu_k_lens=cu_k, **kw)
+        heads = [h for h in range(case.num_q_heads) if int(case.head_mask[h])]
+        kvh = len({h // (case.num_q_heads // case.num_kv_heads) for h in heads})
+        alg_bytes = k_out.numel() * 2 + case.kv_tokens() * kvh * case.head_dim * 2 + 2 * q_out.numel() * 2
+        tokens, launches, kernel = case.kv_tokens(), 2, "capture_k_kernel (+ capture_q_kernel)"
+        host_k = torch.empty(k_out.shape, dtype=torch.bfloat16).pin_memory()
+
+        def e2e():
+            _, k, _ = step()
+            host_k.copy_(k, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+        h2d, d2h = 0, k_out.numel() * 2
+
+    def timed(fn, n):
+        for _ in range(args.warmup):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / 1e3 / n
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    t = timed(step, args.steps)
+    clocks = sampler.stop()
+    t_e2e = timed(e2e, max(5, min(args.steps, 50)))
+    peaks = load_peaks()
+    achieved = alg_bytes / t / 1e9
+    print(json.dumps({
+        "metric": METRIC, "value": tokens / t, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}", "l2": "inputs larger than L2"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": f"of {peaks['source']}",
+                     "kernel": kernel, "algorithmic_bytes": alg_bytes},
+        "e2e": {"value": tokens / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": t_e2e * 1e3},
+        "gpu_launches": launches * args.steps,
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
 def run_mixed(args):
     """The mixed chunked batch: one decode call (256 sequences) and one prefill call (2 chunks of 2048
     rows) per step.  The decode call is HBM-bound and the prefill call tensor-bound, so the step issues
@@ -319,6 +395,9 @@ def main():
         raise SystemExit(f"unknown workload {args.workload}; choose from {sorted(WORKLOADS)}")
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.workload in ("steer_residual", "capture_qk"):
+        run_extra(args)
         return
     if args.workload == "cfg4_mixed":
         if int(os.environ.get("WORLD_SIZE", "1")) > 1:

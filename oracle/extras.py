@@ -2,7 +2,9 @@
 the analyzer's score reduction, residual-stream steering and the raw q/k capture.  fp64 where
 floating point is involved, plain indexing where bytes are moved.  Shares nothing with the CUDA code.
 
-Readings where the paper is silent (its analyzer body is elided): `mean` averages the span masses
+`scores`: parity unpinned against the paper -- its analyzer body is elided, so the formula below is a
+reading of the paper's words; the arithmetic of that reading is pinned by closed forms and brute force.
+Readings where the paper is silent: `mean` averages the span masses
 over the probed heads; `sum_normalize` first divides every head's span masses by that head's total
 over the configured spans (instruction mass / (instruction + data mass) for two spans) and then
 averages over the heads; a head whose total is zero contributes zero.

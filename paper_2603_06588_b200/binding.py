@@ -236,17 +236,23 @@ class HookAttn:
         return hidden
 
     def hook_capture_qk(self, is_decode: bool, *, q, k_cache, v_cache, block_table, seq_lens, cu_q_lens=None,
-                        head_mask=None, probe_rows=HOOK_PROBE_ROWS_ALL, status=None, stream=None, **_ignored):
-        """Raw q/k capture of the probed heads.  Returns ``(q_out [rows, P, D], k_out [sum L, P, D], cu_k_lens)``."""
+                        head_mask=None, probe_rows=HOOK_PROBE_ROWS_ALL, status=None, stream=None,
+                        q_out=None, k_out=None, cu_k_lens=None, **_ignored):
+        """Raw q/k capture of the probed heads.  Returns ``(q_out [rows, P, D], k_out [sum L, P, D], cu_k_lens)``.
+        The three outputs are allocated (and the prefix sums computed, with one host sync for the total)
+        unless the caller passes them."""
         nprobed = 0 if head_mask is None else int((head_mask != 0).sum())
         total_q, hq, d = q.shape
         last_only = is_decode or probe_rows == HOOK_PROBE_ROWS_LAST
         rows = int(seq_lens.shape[0]) if last_only else int(total_q)
-        cu_k = torch.zeros(seq_lens.shape[0] + 1, dtype=torch.int32, device=q.device)
-        cu_k[1:] = torch.cumsum(seq_lens, 0)
-        total_k = int(cu_k[-1].item())
-        q_out = torch.zeros((rows, nprobed, d), dtype=torch.bfloat16, device=q.device)
-        k_out = torch.zeros((total_k, nprobed, d), dtype=torch.bfloat16, device=q.device)
+        cu_k = cu_k_lens
+        if cu_k is None:
+            cu_k = torch.zeros(seq_lens.shape[0] + 1, dtype=torch.int32, device=q.device)
+            cu_k[1:] = torch.cumsum(seq_lens, 0)
+        if q_out is None:
+            q_out = torch.zeros((rows, nprobed, d), dtype=torch.bfloat16, device=q.device)
+        if k_out is None:
+            k_out = torch.zeros((int(cu_k[-1].item()), nprobed, d), dtype=torch.bfloat16, device=q.device)
         p, keep = make_params(q=q, k_cache=k_cache, v_cache=v_cache, block_table=block_table, seq_lens=seq_lens,
                               cu_q_lens=cu_q_lens, head_mask=head_mask, probe_rows=probe_rows, status=status)
         rc = int(self._lib.hook_capture_qk(self._h, ctypes.byref(p), int(bool(is_decode)), q_out.data_ptr(),

@@ -106,15 +106,29 @@ __global__ void __launch_bounds__(256) capture_k_kernel(const KernelArgs a, cons
     const int rows_per_step = 256 / LPR;
     const int32_t* bt = a.block_table + (int64_t)s * a.max_blocks;
     const int64_t out0 = (int64_t)cu_k[s] + t0;
-    for (int r = sub; r < nkeys * a.P; r += rows_per_step) {
-        const int tk = r / a.P, pi = r % a.P;
-        const int t = t0 + tk;
-        int page = bt[t / kPage];
-        if (page < 0 || page >= a.num_blocks) { report(a.status, HOOK_ATTN_ERR_BOUNDS); continue; }
-        const int kvh = sh_heads[pi] / a.G;
-        const uint4 v = *reinterpret_cast<const uint4*>(a.k + (int64_t)page * a.bs + (int64_t)(t % kPage) * a.ts +
+    // four rows per thread and step: the loads are issued together, then the stores
+    const int total = nkeys * a.P;
+    for (int r0 = sub; r0 < total; r0 += 4 * rows_per_step) {
+        uint4 v[4];
+        int64_t dst[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int r = r0 + u * rows_per_step;
+            dst[u] = -1;
+            if (r < total) {
+                const int tk = r / a.P, pi = r % a.P;
+                const int t = t0 + tk;
+                const int page = bt[t / kPage];
+                if (page < 0 || page >= a.num_blocks) { report(a.status, HOOK_ATTN_ERR_BOUNDS); continue; }
+                const int kvh = sh_heads[pi] / a.G;
+                v[u] = *reinterpret_cast<const uint4*>(a.k + (int64_t)page * a.bs + (int64_t)(t % kPage) * a.ts +
                                                        (int64_t)kvh * a.hs + part * 8);
-        *reinterpret_cast<uint4*>(k_out + ((out0 + tk) * a.P + pi) * HD + part * 8) = v;
+                dst[u] = ((out0 + tk) * a.P + pi) * HD + part * 8;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (dst[u] >= 0) *reinterpret_cast<uint4*>(k_out + dst[u]) = v[u];
     }
 }
 
