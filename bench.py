@@ -497,23 +497,39 @@ def main():
     # end to end through the public call with host buffers: the step's inputs (queries, tables,
     # lengths, spans) come from pinned host memory and the results go back to the host every step;
     # the KV cache is state that stays resident on the device, like it does while serving.
-    host_in = {k: kw[k].cpu().pin_memory() for k in ("q", "block_table", "seq_lens", "cu_q_lens", "spans") if k in kw}
-    dev_in = {k: torch.empty_like(kw[k]) for k in host_in}
-    host_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
-    host_mass = None if mass is None else torch.empty(mass.shape, dtype=mass.dtype).pin_memory()
+    # The step's inputs are packed into one pinned host buffer and one device buffer (256-byte aligned
+    # views), the results into one device buffer and one pinned host buffer: one copy each way.
+    dev_str = f"cuda:{local}"
+
+    def pack(tensors, device, pin=False):
+        offs, total = {}, 0
+        for k, t in tensors.items():
+            offs[k] = total
+            total += (t.numel() * t.element_size() + 255) // 256 * 256
+        buf = torch.empty(total, dtype=torch.uint8, device=device)
+        if pin:
+            buf = buf.pin_memory()
+        views = {k: buf[offs[k]:offs[k] + t.numel() * t.element_size()].view(t.dtype).view(t.shape) for k, t in tensors.items()}
+        return buf, views
+
+    step_in = {k: kw[k] for k in ("q", "block_table", "seq_lens", "cu_q_lens", "spans") if k in kw}
+    host_in_buf, host_in = pack(step_in, "cpu", pin=True)
+    for k, t in step_in.items():
+        host_in[k].copy_(t)
+    dev_in_buf, dev_in = pack(step_in, dev_str)
+    step_out = {"out": out} if mass is None else {"out": out, "mass": mass}
+    dev_out_buf, dev_out = pack(step_out, dev_str)
+    host_out_buf, _host_out = pack(step_out, "cpu", pin=True)
     e2e_kw = dict(kw)
     e2e_kw.update(dev_in)
-    plan_e2e = eng.plan(case.is_decode, out=out, span_mass=mass, **e2e_kw)
-    h2d = sum(t.numel() * t.element_size() for t in host_in.values())
-    d2h = host_out.numel() * host_out.element_size() + (0 if host_mass is None else host_mass.numel() * 4)
+    plan_e2e = eng.plan(case.is_decode, out=dev_out["out"], span_mass=dev_out.get("mass"), **e2e_kw)
+    h2d = sum(t.numel() * t.element_size() for t in step_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in step_out.values())
 
     def e2e_step():
-        for k, t in host_in.items():
-            dev_in[k].copy_(t, non_blocking=True)
+        dev_in_buf.copy_(host_in_buf, non_blocking=True)
         plan_e2e.run()
-        host_out.copy_(out, non_blocking=True)
-        if host_mass is not None:
-            host_mass.copy_(mass, non_blocking=True)
+        host_out_buf.copy_(dev_out_buf, non_blocking=True)
         torch.cuda.current_stream().synchronize()
 
     n_e2e = max(10, min(args.steps, 500))
