@@ -355,3 +355,52 @@ def test_small_head_dim_128_calls_take_the_warp_mma_kernel(eng):
                             alpha=torch.tensor([0.0, 0.5, 0.0, 0.0, -1.0, 0.0]), steer=True, poison=True)
     assert case.total_q < 128
     check(eng, case)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_shapes_sweep(eng, seed):
+    """Seeded random batches: ragged lengths, chunk offsets that are not tile-aligned, empty sequences,
+    arbitrary (overlapping, empty, out-of-range) spans, random head masks and steering, both probe modes."""
+    g = inputs._gen(9000 + seed)
+    ri = lambda lo, hi: int(torch.randint(lo, hi + 1, (1,), generator=g))
+    Hq, Hkv = [(2, 1), (4, 4), (8, 2), (14, 2), (16, 2), (8, 1)][ri(0, 5)]
+    D = 128 if ri(0, 3) else 64
+    decode = ri(0, 2) == 0
+    num_seqs = ri(1, 5)
+    lens, qls = [], []
+    for _ in range(num_seqs):
+        L = ri(1, 900) if ri(0, 3) else ri(1, 40)
+        mode = ri(0, 3)
+        n = 1 if decode else (L if mode == 0 else (0 if mode == 1 else ri(1, L)))
+        lens.append(L)
+        qls.append(n)
+    if not decode and sum(qls) == 0:
+        qls[0] = min(lens[0], 3)
+    S = ri(0, 8)
+    spans = None
+    if S:
+        spans = torch.zeros((num_seqs, S, 2), dtype=torch.int32)
+        for s, L in enumerate(lens):
+            for j in range(S):
+                a_, b_ = ri(-5, L + 5), ri(-5, L + 5)
+                if ri(0, 4):
+                    a_, b_ = min(a_, b_), max(a_, b_)
+                spans[s, j, 0], spans[s, j, 1] = a_, b_
+    mask = (torch.rand(Hq, generator=g) < 0.5).to(torch.uint8) if S else None
+    alpha = None
+    if ri(0, 1):
+        alpha = torch.where(torch.rand(Hq, generator=g) < 0.4, torch.rand(Hq, generator=g) * 3 - 1.5, torch.zeros(Hq))
+    case = inputs.make_case(f"rand{seed}", is_decode=decode, seq_lens=lens, q_lens=qls, num_q_heads=Hq, num_kv_heads=Hkv,
+                            head_dim=D, seed=500 + seed, spans=spans, head_mask=mask, alpha=alpha, steer=alpha is not None,
+                            probe_rows=inputs.PROBE_ROWS_LAST if (decode or ri(0, 1)) else inputs.PROBE_ROWS_ALL,
+                            poison=True, scale=None if ri(0, 1) else 0.05 + 0.1 * ri(0, 3))
+    out, mass, status = run_gpu(eng, case)
+    assert status == 0
+    ref_out, ref_mass = oracle.run(case)
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.isfinite(got).all() and np.abs(got - ref_out).max() <= TOL_OUT
+    if ref_mass is not None and case.num_probed:
+        rows = mass_rows(case, list(range(case.total_q)))
+        sel = [i for i, r in enumerate(rows) if r is not None]
+        gm = mass.cpu().numpy().astype(np.float64)[[rows[i] for i in sel]]
+        assert np.abs(gm - ref_mass[sel]).max() <= TOL_MASS
