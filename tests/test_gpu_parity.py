@@ -398,7 +398,10 @@ def test_random_shapes_sweep(eng, seed):
     assert status == 0
     ref_out, ref_mass = oracle.run(case)
     got = out.float().cpu().numpy().astype(np.float64)
-    assert np.isfinite(got).all() and np.abs(got - ref_out).max() <= TOL_OUT
+    # 2e-2 covers bf16 rounding (spacing 2^-6 below 4) plus the arithmetic; outputs in [4, 8) sit on a
+    # grid of 2^-5, whose half step alone is 2^-6, so that much is added there
+    tol = np.where(np.abs(ref_out) < 4.0, TOL_OUT, TOL_OUT + 2.0 ** -6)
+    assert np.isfinite(got).all() and np.all(np.abs(got - ref_out) <= tol) and np.abs(ref_out).max() < 8.0
     if ref_mass is not None and case.num_probed:
         rows = mass_rows(case, list(range(case.total_q)))
         sel = [i for i, r in enumerate(rows) if r is not None]
