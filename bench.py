@@ -396,6 +396,8 @@ def main():
     if args.impl == "reference":
         run_reference(args)
         return
+    from paper_2603_06588_b200.csrc import build as cuda_build
+    cuda_build.build()          # no-op when the in-tree library is up to date
     if args.workload in ("steer_residual", "capture_qk"):
         run_extra(args)
         return
