@@ -397,7 +397,8 @@ def main():
         run_reference(args)
         return
     from paper_2603_06588_b200.csrc import build as cuda_build
-    cuda_build.build()          # no-op when the in-tree library is up to date
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        cuda_build.build()      # no-op when the in-tree library is up to date
     if args.workload in ("steer_residual", "capture_qk"):
         run_extra(args)
         return
