@@ -40,6 +40,7 @@ UNIT = "tokens/s"
 WORKLOADS = {
     "cfg2_decode": "decode batch: 64 seqs x 1 token, ctx U[512,4096], Hq32/Hkv8, D128, 16 probed heads, 2 spans, 4 steered heads",
     "cfg3_prefill": "prefill: 8 seqs x 4096 tokens causal, Hq32/Hkv8, D128, ~10% (layer,head) pairs probed, 3 spans, one layer call per step",
+    "cfg3_prefill_32layers": "prefill: 32 independent layers' worth of seeded inputs (8 seqs x 4096 each), the seeded 10% of the 1024 (layer, head) pairs probed, 3 spans; one step = 32 layer calls",
     "cfg3_prefill_small": "prefill, profiling size: 2 seqs x 2048 tokens causal, Hq32/Hkv8, D128, layer-0 probes, 3 spans",
     "cfg4_decode": "mixed batch, decode part: 256 seqs, ctx U[1024,8192], Hq28/Hkv4, D128, 14 probed heads, 4 spans, 8 steered heads",
     "cfg4_prefill": "mixed batch, prefill part: 2 chunks of 2048 tokens on 4096-token contexts, Hq28/Hkv4, D128",
@@ -288,6 +289,62 @@ def run_extra(args):
 
 
 # ------------------------------------------------------------------------------------------------
+def run_layers(args):
+    """The 32-layer prefill workload: every layer has its own seeded q/K/V, block table, spans and head
+    mask (layers without a probed head run with hooks off).  One step = 32 layer calls back to back."""
+    from paper_2603_06588_b200 import binding
+    args.warmup = max(args.warmup, 3)
+    torch.cuda.set_device(0)
+    eng = binding.HookAttn(0)
+    plans, flops, tokens, probed = [], 0.0, 0, 0
+    for layer in range(args.layers):
+        case = inputs.config3_prefill(layer=layer)
+        if case.num_probed == 0:
+            case = case.without_hooks()
+        probed += case.num_probed
+        plans.append(eng.plan(False, **binding.case_to_device(case)))
+        flops += algorithmic_work(case)[1]
+        tokens = case.total_q
+    for p in plans:
+        p.run()
+    torch.cuda.synchronize()
+
+    def step():
+        for p in plans:
+            p.run()
+
+    for _ in range(args.warmup):
+        step()
+    sampler = ClockSampler(0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    t = e0.elapsed_time(e1) / 1e3 / args.steps
+    peaks = load_peaks()
+    peak = peaks["bf16_tflops"] if t * args.steps < 2.0 else peaks["bf16_tflops_sustained"]
+    achieved = flops / t / 1e12
+    print(json.dumps({
+        "metric": METRIC, "value": tokens * args.layers / t, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "ms_per_layer_call": t * 1e3 / args.layers,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"cfg3_prefill_32layers: {WORKLOADS['cfg3_prefill_32layers']}", "layers": args.layers,
+                   "probed_layer_head_pairs": probed, "l2": "inputs larger than L2 (0.67 GB per layer call)"},
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "traffic": None, "peak_source": f"of {peaks['source']}", "kernel": "prefill_tc_kernel",
+                     "algorithmic_flops": flops, "frac_of_datasheet": achieved / 2250.0},
+        "e2e": None, "gpu_launches": args.layers * args.steps,
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"], "power_w": clocks["power_w"]},
+    }))
+
+
+# ------------------------------------------------------------------------------------------------
 def run_mixed(args):
     """The mixed chunked batch: one decode call (256 sequences) and one prefill call (2 chunks of 2048
     rows) per step.  The decode call is HBM-bound and the prefill call tensor-bound, so the step issues
@@ -390,6 +447,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-budget", type=float, default=2.0, help="seconds of CPU time per oracle step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=32, help="layers of the cfg3_prefill_32layers workload")
     args = ap.parse_args()
     if args.workload not in WORKLOADS:
         raise SystemExit(f"unknown workload {args.workload}; choose from {sorted(WORKLOADS)}")
@@ -399,6 +457,9 @@ def main():
     from paper_2603_06588_b200.csrc import build as cuda_build
     if int(os.environ.get("LOCAL_RANK", "0")) == 0:
         cuda_build.build()      # no-op when the in-tree library is up to date
+    if args.workload == "cfg3_prefill_32layers":
+        run_layers(args)
+        return
     if args.workload in ("steer_residual", "capture_qk"):
         run_extra(args)
         return
