@@ -126,8 +126,9 @@ size_t hook_attn_workspace_bytes(const hook_attn_params* p, int is_decode);
  * (Section 2.2 recompute + Section 2 steering, fused into the attention forward.) */
 int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
 
-/* Decode: exactly one query row per sequence (total_q == num_seqs, cu_q_lens ignored); keys are
- * split into chunks that are reduced independently and merged in a fixed order, so results are
+/* Decode: exactly one query row per sequence (total_q == num_seqs, cu_q_lens ignored).  The keys
+ * of all sequences are dealt out in equal shares to a fixed number of workers; each share is
+ * reduced independently and the pieces of a sequence are merged in a fixed order, so results are
  * bit-identical from run to run.  span_mass has one row per sequence. */
 int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
 

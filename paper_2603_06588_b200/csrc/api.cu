@@ -11,8 +11,8 @@ namespace hook_attn {
 // decode.cu
 cudaError_t configure_decode();
 cudaError_t launch_decode(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st);
-size_t decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim, int max_chunks);
-int decode_pick_chunk(int num_seqs, int Hkv, int max_blocks, int num_sms);
+size_t decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim, int max_blocks);
+int decode_workers(int num_seqs, int Hkv, int head_dim, int max_blocks);
 // prefill_mma.cu
 cudaError_t configure_prefill_mma();
 cudaError_t launch_prefill_mma(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st);
@@ -40,8 +40,6 @@ struct hook_attn_handle {
 };
 
 namespace {
-
-constexpr int kDefaultSMs = 148;
 
 int validate_common(const hook_attn_params* p, bool decode)
 {
@@ -159,9 +157,7 @@ size_t hook_attn_workspace_bytes(const hook_attn_params* p, int is_decode)
     if (validate_common(p, is_decode != 0) != HOOK_ATTN_OK) return 0;
     if (!is_decode) return 0;
     const int G = p->num_q_heads / p->num_kv_heads;
-    const int chunk = decode_pick_chunk(p->num_seqs, p->num_kv_heads, p->max_blocks_per_seq, kDefaultSMs);
-    const int max_chunks = (p->max_blocks_per_seq * kPage + chunk - 1) / chunk;
-    return decode_workspace_bytes(p->num_seqs, p->num_kv_heads, G, p->head_dim, max_chunks > 0 ? max_chunks : 1);
+    return decode_workspace_bytes(p->num_seqs, p->num_kv_heads, G, p->head_dim, p->max_blocks_per_seq);
 }
 
 int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream)
@@ -190,9 +186,8 @@ int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* 
     if (rc != HOOK_ATTN_OK) return rc;
     if (p->num_seqs > 0 && p->max_blocks_per_seq == 0) return HOOK_ATTN_ERR_INVALID_ARG;
     if (p->num_seqs == 0) return handle ? HOOK_ATTN_OK : HOOK_ATTN_ERR_INVALID_ARG;
-    a.chunk = decode_pick_chunk(p->num_seqs, p->num_kv_heads, p->max_blocks_per_seq, kDefaultSMs);
-    a.max_chunks = (p->max_blocks_per_seq * kPage + a.chunk - 1) / a.chunk;
-    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, a.max_chunks);
+    a.workers = decode_workers(p->num_seqs, p->num_kv_heads, p->head_dim, p->max_blocks_per_seq);
+    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, p->max_blocks_per_seq);
     if (!p->workspace || p->workspace_bytes < need) return HOOK_ATTN_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(p->workspace) & 15u) return HOOK_ATTN_ERR_WORKSPACE;
     if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
@@ -245,9 +240,8 @@ int hook_attn_decode_static_scratch(hook_attn_handle* handle, const hook_attn_pa
     if (rc != HOOK_ATTN_OK) return rc;
     if (p->num_seqs > 0 && p->max_blocks_per_seq == 0) return HOOK_ATTN_ERR_INVALID_ARG;
     if (p->num_seqs == 0) return handle ? HOOK_ATTN_OK : HOOK_ATTN_ERR_INVALID_ARG;
-    a.chunk = decode_pick_chunk(p->num_seqs, p->num_kv_heads, p->max_blocks_per_seq, kDefaultSMs);
-    a.max_chunks = (p->max_blocks_per_seq * kPage + a.chunk - 1) / a.chunk;
-    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, a.max_chunks);
+    a.workers = decode_workers(p->num_seqs, p->num_kv_heads, p->head_dim, p->max_blocks_per_seq);
+    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, p->max_blocks_per_seq);
     if (need > HOOK_ATTN_STATIC_SCRATCH_BYTES) return HOOK_ATTN_ERR_WORKSPACE;   // batch too large for the fixed array
     if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
     int current = -1;
@@ -256,7 +250,7 @@ int hook_attn_decode_static_scratch(hook_attn_handle* handle, const hook_attn_pa
     float* scratch = nullptr;
     rc = static_scratch_address(handle->device, &scratch);
     if (rc != HOOK_ATTN_OK) return rc;
-    a.ws = scratch;   // every partial the merge reads is written by the split-K kernel of the same call:
+    a.ws = scratch;   // every partial the merge reads is written by the streaming kernel of the same call:
                       // nothing in the array has to start at zero, stale contents are never read
     cudaError_t e = launch_decode(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;

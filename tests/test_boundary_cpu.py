@@ -126,9 +126,11 @@ def test_decode_shape_and_workspace_checks(lib):
 
 
 def test_workspace_scales_with_the_bounds(lib):
+    # one partial per (sequence, KV head) plus one per worker of the fixed grid
     a = lib.hook_attn_workspace_bytes(ctypes.byref(_params(num_seqs=4, total_q=4)), 1)
     b = lib.hook_attn_workspace_bytes(ctypes.byref(_params(num_seqs=8, total_q=8)), 1)
-    assert b == 2 * a
+    c = lib.hook_attn_workspace_bytes(ctypes.byref(_params(num_seqs=12, total_q=12)), 1)
+    assert a > 0 and c - b == b - a > 0
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="only meaningful without a GPU")

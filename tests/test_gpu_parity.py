@@ -128,6 +128,41 @@ def test_decode_shapes_and_ragged_lengths(eng, Hq, Hkv, D):
     check(eng, case)
 
 
+def test_decode_page_shares_many_and_skewed_sequences(eng):
+    """The decode kernel deals the pages of all sequences out to its workers in equal shares.  Here: more
+    sequences than one window of its page-count scan (1024), lengths from one key to hundreds of pages, two
+    long sequences that many workers share, workers whose share crosses dozens of short sequences, and
+    then the same batch with empty sequences in the middle (reported, zero-filled, the rest untouched)."""
+    g = inputs._gen(4242)
+    lens = torch.randint(1, 40, (1300,), generator=g).tolist()
+    lens[7], lens[1100] = 9000, 5000
+    alpha = torch.zeros(4)
+    alpha[1] = -0.6
+    case = inputs.make_case("dec_many", is_decode=True, seq_lens=lens, q_lens=[1] * len(lens), num_q_heads=4,
+                            num_kv_heads=2, head_dim=64, seed=4243, num_spans=2,
+                            head_mask=torch.tensor([1, 0, 1, 1], dtype=torch.uint8), alpha=alpha, steer=True,
+                            probe_rows=inputs.PROBE_ROWS_LAST, poison=True)
+    check(eng, case)
+    out0, mass0, _ = run_gpu(eng, case)
+    holes = list(lens)
+    for i in (3, 1023, 1024, 1200):
+        holes[i] = 0
+    out1, mass1, st = run_gpu(eng, inputs.with_seq_lens(case, holes))
+    assert st == binding.HOOK_ATTN_ERR_INVALID_ARG
+    keep = torch.tensor([i not in (3, 1023, 1024, 1200) for i in range(len(lens))], device=out0.device)
+    assert torch.all(out1[~keep] == 0) and torch.all(mass1[~keep] == 0)
+    assert (out1[keep].float() - out0[keep].float()).abs().max().item() <= TOL_OUT
+    assert (mass1[keep] - mass0[keep]).abs().max().item() <= TOL_MASS
+
+
+def test_decode_fewer_pages_than_workers(eng):
+    case = inputs.make_case("dec_three_pages", is_decode=True, seq_lens=[1, 17], q_lens=[1, 1], num_q_heads=2,
+                            num_kv_heads=1, head_dim=128, seed=5, num_spans=2,
+                            head_mask=torch.tensor([1, 1], dtype=torch.uint8), probe_rows=inputs.PROBE_ROWS_LAST,
+                            poison=True)
+    check(eng, case)
+
+
 @pytest.mark.parametrize("Hq,Hkv,D", [(8, 8, 64), (4, 1, 64), (14, 2, 128), (8, 2, 128)])
 def test_prefill_shapes_ragged_and_chunked(eng, Hq, Hkv, D):
     seq_lens = [1, 17, 64, 65, 130, 300, 77, 200]
