@@ -9,11 +9,14 @@
 //              running reference maximum moves, and runs the epilogue of tile A;
 //   warps 4-7  the same for tile B;
 //   warp  8    producer: resolves pages through the block table and issues one TMA box load per
-//              (page, 64-wide half of the head) into 128B-swizzled K and V stages;
-//   warp  9    owns tensor memory and issues the MMAs: S = Q K^T (both operands K-major in shared
-//              memory) and O += P V (P from tensor memory, V as the MN-major B operand), ordered
-//              PV(A,j) QK(A,j+1) PV(B,j) QK(B,j+1) so that one tile's softmax overlaps the other
-//              tile's tensor work.
+//              (page, 64-wide half of the head) into 128B-swizzled K and V stages; it also zeroes the
+//              value rows past the end of the sequence in the last tile;
+//   warp  9    owns tensor memory; one elected thread of it issues the MMAs: S = Q K^T (both operands
+//              K-major in shared memory) and O += P V (P from tensor memory, V as the MN-major B
+//              operand), ordered PV(A,j) QK(A,j+1) PV(B,j) QK(B,j+1) so that one tile's softmax
+//              overlaps the other tile's tensor work.  That thread is the pacemaker of the CTA, so
+//              it does nothing else: the K/V stages are handed back to the producer by a softmax
+//              thread of the later tile, which sees the completion of QK(.,j) anyway.
 // Tensor memory (512 columns): S_A/P_A at 0, S_B/P_B at 128, O_A at 256, O_B at 384.
 //
 // The softmax keeps a *reference* maximum that is only raised when a tile's maximum exceeds it by
@@ -45,6 +48,19 @@ constexpr int kStages = 2;
 constexpr int kSmemBytes = 2 * kTileBytes + 2 * kStages * kTileBytes + 1024;   // Q(A,B) + K,V stages + alignment slack
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;       // log2 units
+// Of every eight pairs of probabilities, this many are computed with a polynomial on the FMA pipe
+// instead of the special-function unit (which gives 16 results per clock and SM and would otherwise
+// set the pace of the softmax).
+#ifndef HOOK_TC_POLY_PER8
+#define HOOK_TC_POLY_PER8 0
+#endif
+constexpr int kPolyPer8 = HOOK_TC_POLY_PER8;
+// The probabilities of a tile are handed to the MMA thread in two halves of 64 keys, so that P V of
+// the first half runs while the second half is still being exponentiated.
+#ifndef HOOK_TC_SPLIT_P
+#define HOOK_TC_SPLIT_P 0
+#endif
+constexpr bool kSplitP = HOOK_TC_SPLIT_P != 0;
 constexpr int kMaskTiles = 1024;                // key tiles with a precomputed span classification
 
 // Which spans does key tile [k0, k0 + 128) touch?  Low byte: spans that contain the whole tile;
@@ -196,6 +212,25 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
+// 2^x for a pair of arguments x <= 8 on the FMA pipe: x = n + f with n = round(x) (magic-number
+// add), 2^f on [-1/2, 1/2] from a degree-4 polynomial (relative error 3e-6), 2^n added into the
+// exponent field.  Arguments below -126 (masked keys are -inf) give a value below 1e-37.
+__device__ __forceinline__ float2 poly_exp2(float2 x)
+{
+    const float kMagic = 12582912.f;   // 1.5 * 2^23: the sum's low mantissa bits are round(x)
+    x.x = fmaxf(x.x, -126.f);
+    x.y = fmaxf(x.y, -126.f);
+    const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
+    const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
+    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
+    float2 p = make_float2(0.00957401655614376f, 0.00957401655614376f);
+    p = __ffma2_rn(p, f, make_float2(0.055918190628290176f, 0.055918190628290176f));
+    p = __ffma2_rn(p, f, make_float2(0.2402464896440506f, 0.2402464896440506f));
+    p = __ffma2_rn(p, f, make_float2(0.6931217312812805f, 0.6931217312812805f));
+    p = __ffma2_rn(p, f, make_float2(0.9999992847442627f, 0.9999992847442627f));
+    return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),
+                       __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
@@ -219,6 +254,8 @@ struct Barriers {
     uint64_t q_full[2];
     uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
     uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t p_half[2];       // the first 64 keys' probabilities of a tile are in tensor memory
+    uint64_t v_tail;          // the producer has zeroed the value rows past the end of the sequence
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -286,6 +323,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             mbar_init(smem_u32(&bars.q_full[x]), 1);
             mbar_init(smem_u32(&bars.s_full[x]), 1);
             mbar_init(smem_u32(&bars.p_full[x]), 128);
+            mbar_init(smem_u32(&bars.p_half[x]), 128);
             mbar_init(smem_u32(&bars.o_full[x]), 1);
         }
         for (int i = 0; i < kStages; ++i) {
@@ -294,6 +332,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             mbar_init(smem_u32(&bars.v_full[i]), 1);
             mbar_init(smem_u32(&bars.v_empty[i]), 1);
         }
+        mbar_init(smem_u32(&bars.v_tail), 1);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -363,6 +402,25 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
                 }
             }
         }
+        if (ok && nmax > 0 && nmax * kBN > L) {
+            // value rows at keys >= L (page tails, pages that were never loaded) must not reach the
+            // tensor cores: 0 * NaN would poison the accumulator.  Zero them in shared memory once the
+            // last tile has landed, then tell the MMA thread.
+            const int j = nmax - 1, st = j & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1));
+            if (ok) {
+                const int r_first = L - j * kBN;
+                const uint32_t vb = sV + st * kTileBytes;
+                for (int idx = lane; idx < (kBN - r_first) * 16; idx += 32) {
+                    const int r = r_first + (idx >> 4), c = idx & 15;
+                    const uint32_t addr = vb + (c >> 3) * kHalfBytes + r * 128 + (c & 7) * 16;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.v_tail));
+            }
+        }
     } else if (warp == kMmaWarp) {
         // ================================ MMA issue ================================
         constexpr uint32_t idesc_qk = instr_desc(0), idesc_pv = instr_desc(1);
@@ -381,70 +439,46 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             }
             tc_commit(smem_u32(&bars.s_full[x]));
         };
-        auto issue_pv = [&](int x, int j) {
+        auto issue_pv = [&](int x, int j, int ks0, int ks1) {
             const uint64_t dv = (j & 1) ? dV[1] : dV[0];
 #pragma unroll
-            for (int ks = 0; ks < kBN / 16; ++ks)
+            for (int ks = ks0; ks < ks1; ++ks)
                 tc_mma_ts(tO[x], tS[x] + ks * 8, desc_advance(dv, (ks * 16 * 128) >> 4), idesc_pv, (ks > 0) || (j > 0));
         };
+        if (lane == 0) {
+            // one thread runs the whole issue loop: no votes, no warp barriers on the pacemaker's path
 #pragma unroll
-        for (int x = 0; x < 2; ++x)
-            if (ok && ntiles[x] > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_full[x]), 0));
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.k_full[0]), 0));
-        if (ok) {
-            tc_fence_after();
-            if (lane == 0) {
+            for (int x = 0; x < 2; ++x)
+                if (ok && ntiles[x] > 0) ok = mbar_wait(smem_u32(&bars.q_full[x]), 0);
+            if (ok) ok = mbar_wait(smem_u32(&bars.k_full[0]), 0);
+            if (ok) {
+                tc_fence_after();
                 if (ntiles[0] > 0) issue_qk(0, 0);
                 if (ntiles[1] > 0) issue_qk(1, 0);
-                if (kStages < nmax) tc_commit(smem_u32(&bars.k_empty[0]));   // only if the producer will wait for it
             }
-            __syncwarp();
-        }
-        for (int j = 0; j < nmax && ok; ++j) {
-            const int st = j & 1;
-            const uint32_t ph = (j >> 1) & 1;
-            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_full[st]), ph));
-            if (!ok) break;
-            if (j == nmax - 1 && (j + 1) * kBN > L) {
-                // value rows at keys >= L (page tails, pages that were never loaded) must not reach the
-                // tensor cores: 0 * NaN would poison the accumulator.  Zero them in shared memory.
-                const int r_first = L - j * kBN;
-                const uint32_t vb = sV + st * kTileBytes;
-                for (int idx = lane; idx < (kBN - r_first) * 16; idx += 32) {
-                    const int r = r_first + (idx >> 4), c = idx & 15;
-                    const uint32_t addr = vb + (c >> 3) * kHalfBytes + r * 128 + (c & 7) * 16;
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(addr), "r"(0u) : "memory");
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-            }
-            const bool has_next = (j + 1 < nmax);
-            if (has_next) {
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.k_full[(j + 1) & 1]), ((j + 1) >> 1) & 1));
-                if (!ok) break;
-            }
+            for (int j = 0; j < nmax && ok; ++j) {
+                const int st = j & 1;
+                ok = mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1);
+                if (ok && j == nmax - 1 && (j + 1) * kBN > L) ok = mbar_wait(smem_u32(&bars.v_tail), 0);
+                if (ok && j + 1 < nmax) ok = mbar_wait(smem_u32(&bars.k_full[(j + 1) & 1]), ((j + 1) >> 1) & 1);
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                if (j < ntiles[x]) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.p_full[x]), j & 1));
-                    if (!ok) break;
-                    tc_fence_after();
-                    if (lane == 0) {
-                        issue_pv(x, j);
+                for (int x = 0; x < 2; ++x) {
+                    if (ok && j < ntiles[x]) {
+                        if (kSplitP) {
+                            ok = mbar_wait(smem_u32(&bars.p_half[x]), j & 1);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_pv(x, j, 0, kBN / 32);
+                        }
+                        ok = mbar_wait(smem_u32(&bars.p_full[x]), j & 1);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(x, j, kSplitP ? kBN / 32 : 0, kBN / 16);
                         if (j + 1 < ntiles[x]) issue_qk(x, j + 1);
                         else tc_commit(smem_u32(&bars.o_full[x]));
                     }
-                    __syncwarp();
                 }
             }
-            if (!ok) break;
-            if (lane == 0) {
-                // release a stage only if the producer will refill it: an arrive that nobody waits for
-                // could land after the CTA has gone
-                if (j + kStages < nmax) tc_commit(smem_u32(&bars.v_empty[st]));
-                if (j + 1 + kStages < nmax) tc_commit(smem_u32(&bars.k_empty[(j + 1) & 1]));
-            }
-            __syncwarp();
         }
     } else if (warp < 8) {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 208;" ::: "memory");
@@ -454,6 +488,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
         if (nt > 0) {
             const int quarter = warp & 3;
             const int row = quarter * 32 + lane;
+            const bool releases = (nt == nmax) && (x == 1 || ntiles[1] < nmax);   // the tile whose QK is issued last
             const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
             const uint32_t tS = tmem + x * 128 + lane_off;
             const uint32_t tO = tmem + 256 + x * 128 + lane_off;
@@ -468,6 +503,12 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
                 ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), j & 1));
                 if (!ok) break;
                 tc_fence_after();
+                if (releases && (threadIdx.x & 127) == 0) {
+                    // QK(., j) has completed, and with it every MMA issued before it: K tile j and
+                    // V tile j - 1 are free for the producer
+                    mbar_arrive(smem_u32(&bars.k_empty[j & 1]));
+                    if (j > 0) mbar_arrive(smem_u32(&bars.v_empty[(j - 1) & 1]));
+                }
                 const int k0 = j * kBN;
                 const bool need_mask = (k0 + kBN - 1 > first_pos[x]);
 
@@ -530,13 +571,18 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
                     for (int i = 0; i < 16; ++i) {
                         const int e = 32 * c + 2 * i;
                         const float2 xx = __ffma2_rn(make_float2(sc[e], sc[e + 1]), sl2v, nmv);
-                        const float2 pp = make_float2(fast_exp2(xx.x), fast_exp2(xx.y));
+                        const float2 pp = ((i & 7) < kPolyPer8) ? poly_exp2(xx) : make_float2(fast_exp2(xx.x), fast_exp2(xx.y));
                         sc[e] = pp.x;
                         sc[e + 1] = pp.y;
                         rs2[i & 1] = __fadd2_rn(rs2[i & 1], pp);
                         pk[i] = pack_bf16(pp.x, pp.y);
                     }
                     tc_st16(tS + 16 * c, pk);
+                    if (kSplitP && c == 1) {
+                        tc_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(smem_u32(&bars.p_half[x]));
+                    }
                 }
                 const float rs = (rs2[0].x + rs2[0].y) + (rs2[1].x + rs2[1].y);
                 l += rs;
@@ -631,6 +677,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     if (warp == kMmaWarp) {
+        __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
