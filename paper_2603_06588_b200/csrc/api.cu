@@ -12,7 +12,6 @@ namespace hook_attn {
 cudaError_t configure_decode();
 cudaError_t launch_decode(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st);
 size_t decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim, int max_blocks);
-int decode_workers(int num_seqs, int Hkv, int head_dim, int max_blocks);
 // prefill_mma.cu
 cudaError_t configure_prefill_mma();
 cudaError_t launch_prefill_mma(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st);
@@ -186,7 +185,6 @@ int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* 
     if (rc != HOOK_ATTN_OK) return rc;
     if (p->num_seqs > 0 && p->max_blocks_per_seq == 0) return HOOK_ATTN_ERR_INVALID_ARG;
     if (p->num_seqs == 0) return handle ? HOOK_ATTN_OK : HOOK_ATTN_ERR_INVALID_ARG;
-    a.workers = decode_workers(p->num_seqs, p->num_kv_heads, p->head_dim, p->max_blocks_per_seq);
     const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, p->max_blocks_per_seq);
     if (!p->workspace || p->workspace_bytes < need) return HOOK_ATTN_ERR_WORKSPACE;
     if (reinterpret_cast<uintptr_t>(p->workspace) & 15u) return HOOK_ATTN_ERR_WORKSPACE;
@@ -240,7 +238,6 @@ int hook_attn_decode_static_scratch(hook_attn_handle* handle, const hook_attn_pa
     if (rc != HOOK_ATTN_OK) return rc;
     if (p->num_seqs > 0 && p->max_blocks_per_seq == 0) return HOOK_ATTN_ERR_INVALID_ARG;
     if (p->num_seqs == 0) return handle ? HOOK_ATTN_OK : HOOK_ATTN_ERR_INVALID_ARG;
-    a.workers = decode_workers(p->num_seqs, p->num_kv_heads, p->head_dim, p->max_blocks_per_seq);
     const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, p->max_blocks_per_seq);
     if (need > HOOK_ATTN_STATIC_SCRATCH_BYTES) return HOOK_ATTN_ERR_WORKSPACE;   // batch too large for the fixed array
     if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;

@@ -36,7 +36,8 @@ struct KernelArgs {
     float* ws;
     int32_t* status;
     int32_t num_seqs, total_q, Hq, Hkv, G, num_blocks, max_blocks, S, P, probe_rows;
-    int32_t workers;                  // decode: warps of the streaming kernel that share the page list
+    int32_t chunk;                    // decode, fixed chunks: keys per chunk
+    int32_t max_chunks;               // decode, fixed chunks: chunks per sequence the workspace is sized for
     int32_t total_tiles;              // prefill: upper bound on query tiles
     float scale_log2;                 // scale * log2(e)
     bool any_probe, any_steer;

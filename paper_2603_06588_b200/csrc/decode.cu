@@ -1,34 +1,39 @@
 // Split-K decode of the hooked paged attention: one query row per sequence.
 //
-// Kernel 1 (decode_stream): the 16-key pages of all (sequence, KV head) units form one flat list
-// (sequence-major, then KV head, then page); every warp of the grid takes an equal, contiguous share
-// of that list, found from the sequence lengths on the device, so all warps stream the same number
-// of bytes whatever the length mix.  The grid is a small multiple ("rounds") of the two CTAs per SM
-// that fit: one round for short steps, more for long ones, where the hardware's dispatch of later
-// CTAs to whichever SM frees up first evens out the differences in speed.  A warp walks its share
-// unit by unit.  Inside a unit the G <= 8 query heads that share the KV head are
-// processed together with warp-level tensor-core tiles in the transposed orientation: a 16-key
-// page is the M dimension, the query heads are the N = 8 dimension (S^T = K Q^T, O^T = V^T P^T),
-// so no padding work is spent on the single query row.  The warp streams pages through a private
-// multi-stage cp.async pipeline (16-byte copies, zero-filled past the end of the sequence; block
-// ids are fetched 32 at a time), keeps an online softmax per head, and carries the span masses of
-// the probe as extra accumulators in the same frame as the running sum.  At the end of each piece
-// of a unit the warp writes its partial (m, l, o[D], s[S]) to the workspace slot `unit + warp`
-// (both grow along a warp's walk, so the slot is unique).
+// The first kernel reduces pieces of each (sequence, KV head) unit to partials (m, l, o[D], s[S]),
+// the second merges the partials of a unit.  Two ways of cutting the pieces, chosen per call from
+// the batch shape:
 //
-// Kernel 2 (decode_merge): one CTA per (query head, sequence) recomputes which warps covered the
-// unit, merges their partials in warp order (run-to-run bit-identical), normalises, applies the
-// steering add and stores.
+// * decode_splitk (many units): one CTA per (key chunk, KV head, sequence) with a fixed chunk length;
+//   its four warps take the chunk's pages in turn and are merged in shared memory.  With hundreds of
+//   units the hardware's CTA dispatch keeps every SM busy and evens out their speeds.
+// * decode_stream (few units, long sequences): fixed chunks would mean either too few CTAs or many
+//   short ones and a large merge.  Here the 16-key pages of all units form one flat list
+//   (sequence-major, then KV head, then page) and every warp of a grid of two CTAs per SM takes an
+//   equal, contiguous share of it, found from the sequence lengths on the device.  A warp walks its
+//   share unit by unit and writes one partial per unit it touches to slot `unit + warp` (both grow
+//   along the walk, so the slot is unique).
+//
+// Inside a unit the G <= 8 query heads that share the KV head are processed together with
+// warp-level tensor-core tiles in the transposed orientation: a 16-key page is the M dimension, the
+// query heads are the N = 8 dimension (S^T = K Q^T, O^T = V^T P^T), so no padding work is spent on
+// the single query row.  A warp streams pages through a private multi-stage cp.async pipeline
+// (16-byte copies, zero-filled past the end of the sequence), keeps an online softmax per head, and
+// carries the span masses of the probe as extra accumulators in the same frame as the running sum.
+//
+// decode_merge: one CTA per (query head, sequence) folds the unit's partials in a fixed order
+// (run-to-run bit-identical), normalises, applies the steering add and stores.
 #include "common.cuh"
 
 namespace hook_attn {
 
 constexpr int kDecWarps = 4;
 constexpr int kDecStages = 3;
-constexpr int kDecCtas = 2 * 148;                     // one round of the grid: two CTAs on each SM of a B200
-constexpr int kDecMaxRounds = 4;
-constexpr int kScanSeqs = 1024;                       // sequences per window of the page-count scan
+constexpr int kDecCtas = 2 * 148;                     // grid of the streaming kernel: two CTAs on each SM of a B200
+constexpr int kDecWorkers = kDecCtas * kDecWarps;     // its warps, which share the flat page list
+constexpr int kScanSeqs = 512;                        // most sequences the streaming kernel is picked for (a power of two)
 constexpr int kPartPad = 16;   // floats after o[D] in a partial: m, l, s[0..7], padding
+static_assert(kDecCtas <= kScanSeqs, "the streaming kernel is picked for fewer than kDecCtas units");
 
 template <int HD>
 constexpr int decode_smem_bytes()
@@ -46,19 +51,15 @@ __device__ __forceinline__ int decode_pages(int L, int max_blocks)
 }
 
 // Pages of the flat list per worker warp.
-__device__ __forceinline__ long long decode_share(long long flat_total, int workers)
+__device__ __forceinline__ long long decode_share(long long flat_total)
 {
-    return (flat_total + workers - 1) / workers;
+    return (flat_total + kDecWorkers - 1) / kDecWorkers;
 }
 
-// Rounds of the grid, from host-known bounds only (the lengths live on the device): about one round
-// per 2 MB that a CTA would stream if the sequences averaged half of their block tables.
-__host__ inline int decode_rounds(int num_seqs, int Hkv, int head_dim, int max_blocks)
-{
-    const double bytes = 0.5 * num_seqs * Hkv * (double)max_blocks * kPage * head_dim * 2 * 2;
-    const int r = (int)(bytes / (kDecCtas * 2097152.0) + 0.5);
-    return r < 1 ? 1 : (r > kDecMaxRounds ? kDecMaxRounds : r);
-}
+// Bytes at the start of the streaming kernel's workspace that hold the page-count prefix of the
+// sequences (num_seqs + 1 ints, written by its first CTA for the merge kernel).
+__host__ __device__ inline size_t decode_prefix_bytes(int num_seqs) { return (((size_t)num_seqs + 1) * 4 + 255) & ~(size_t)255; }
+
 
 template <int HD, int NS>
 __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const KernelArgs a, const HeadCfg hc)
@@ -71,7 +72,7 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const Ker
     constexpr int EPT = kScanSeqs / (kDecWarps * 32);   // scan entries per thread
 
     extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ int sh_ex[kScanSeqs];                 // page counts, then their exclusive prefix, of one scan window
+    __shared__ int sh_ex[kScanSeqs];                 // page counts of the sequences, then their exclusive prefix
     __shared__ int sh_wsum[kDecWarps];
     __shared__ int sh_span[kDecWarps][2 * kMaxSpans];
 
@@ -79,82 +80,65 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const Ker
     const int g = lane >> 2, tq = lane & 3;
     const int G = a.G;
 
-    // ---- total number of pages (all sequences); the first window's counts stay in shared memory ----
-    int cnt = 0;
-    for (int i = threadIdx.x; i < a.num_seqs; i += kDecWarps * 32) {
-        const int pgs = decode_pages(a.seq_lens[i], a.max_blocks);
-        if (i < kScanSeqs) sh_ex[i] = pgs;
-        cnt += pgs;
+    // ---- exclusive prefix of the page counts (the host only picks this kernel for fewer than
+    //      kScanSeqs sequences); a thread owns EPT consecutive entries ----
+    for (int i = threadIdx.x; i < kScanSeqs; i += kDecWarps * 32)
+        sh_ex[i] = (i < a.num_seqs) ? decode_pages(a.seq_lens[i], a.max_blocks) : 0;
+    __syncthreads();
+    int v[EPT], run = 0;
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) {
+        v[e] = sh_ex[threadIdx.x * EPT + e];
+        run += v[e];
+    }
+    int incl = run;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += t;
+    }
+    if (lane == 31) sh_wsum[warp] = incl;
+    __syncthreads();
+    int off = incl - run, total_pages = 0;
+#pragma unroll
+    for (int w = 0; w < kDecWarps; ++w) {
+        if (w < warp) off += sh_wsum[w];
+        total_pages += sh_wsum[w];
     }
 #pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
-    if (lane == 0) sh_wsum[warp] = cnt;
+    for (int e = 0; e < EPT; ++e) {
+        sh_ex[threadIdx.x * EPT + e] = off;
+        off += v[e];
+    }
     __syncthreads();
-    int total_pages = 0;
-#pragma unroll
-    for (int w = 0; w < kDecWarps; ++w) total_pages += sh_wsum[w];
     // the merge kernel may be scheduled from here on; it waits for this grid's writes itself
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (blockIdx.x == 0) {   // the merge kernel sizes up its unit from this table
+        int* prefix = reinterpret_cast<int*>(a.ws);
+        for (int i = threadIdx.x; i < a.num_seqs; i += kDecWarps * 32) prefix[i] = sh_ex[i];
+        if (threadIdx.x == 0) prefix[a.num_seqs] = total_pages;
+    }
     const long long flat_total = (long long)total_pages * a.Hkv;
-    if (flat_total == 0) return;
-    const long long share = decode_share(flat_total, a.workers);
+    const long long share = decode_share(flat_total);
     const int W = blockIdx.x * kDecWarps + warp;
     const long long f_begin = (long long)W * share;
     const long long f_end = min(f_begin + share, flat_total);
-    const bool has_work = f_begin < f_end;
-    const long long target = f_begin / a.Hkv;   // pages of whole sequences before the start are <= target
-
-    // ---- find the sequence that holds the first page of this warp's share ----
-    int s = -1, ex0 = 0, carry = 0;
-    for (int base = 0; base < a.num_seqs; base += kScanSeqs) {
-        const int nwin = min(kScanSeqs, a.num_seqs - base);
-        __syncthreads();
-        if (base > 0)
-            for (int i = threadIdx.x; i < nwin; i += kDecWarps * 32) sh_ex[i] = decode_pages(a.seq_lens[base + i], a.max_blocks);
-        __syncthreads();
-        // exclusive scan in place: a thread owns EPT consecutive entries
-        int v[EPT], run = 0;
-#pragma unroll
-        for (int e = 0; e < EPT; ++e) {
-            const int i = threadIdx.x * EPT + e;
-            v[e] = (i < nwin) ? sh_ex[i] : 0;
-            run += v[e];
-        }
-        int incl = run;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += t;
-        }
-        __syncthreads();          // sh_wsum of the previous round has been read
-        if (lane == 31) sh_wsum[warp] = incl;
-        __syncthreads();
-        int off = incl - run, wtot = 0;
-#pragma unroll
-        for (int w = 0; w < kDecWarps; ++w) {
-            if (w < warp) off += sh_wsum[w];
-            wtot += sh_wsum[w];
-        }
-#pragma unroll
-        for (int e = 0; e < EPT; ++e) {
-            const int i = threadIdx.x * EPT + e;
-            if (i < nwin) sh_ex[i] = off;
-            off += v[e];
-        }
-        __syncthreads();
-        if (has_work && s < 0 && (long long)carry + wtot > target) {
-            int lo = 0, hi = nwin - 1;      // largest entry whose prefix is <= target
-            while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if ((long long)carry + sh_ex[mid] <= target) lo = mid; else hi = mid - 1;
-            }
-            s = base + lo;
-            ex0 = carry + sh_ex[lo];
-        }
-        carry += wtot;
-    }
-    if (!has_work || s < 0) return;
+    if (f_begin >= f_end) return;
     // from here on the warps are independent: no CTA-wide barrier below
+
+    // ---- the sequence that holds the first page of this warp's share: the last one whose prefix,
+    //      counted in pages of all its KV heads, does not exceed the start ----
+    int s;
+    {
+        const long long target = f_begin / a.Hkv;
+        int lo = 0, hi = a.num_seqs - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (sh_ex[mid] <= target) lo = mid; else hi = mid - 1;
+        }
+        s = lo;
+    }
+    const int ex0 = sh_ex[s];
 
     int L = a.seq_lens[s];
     int np = decode_pages(L, a.max_blocks);
@@ -184,10 +168,14 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const Ker
             __syncwarp();
         }
 
-        int btw = 0;   // block ids of 32 consecutive pages, one per lane
+        // block ids of 32 consecutive pages, one per lane; the next 32 are fetched a window ahead
+        int btw = 0, btw_next = (lane < seg) ? bt[lane] : 0;
         auto issue = [&](int it) {
             if (it < seg) {
-                if ((it & 31) == 0) btw = (it + lane < seg) ? bt[it + lane] : 0;
+                if ((it & 31) == 0) {
+                    btw = btw_next;
+                    btw_next = (it + 32 + lane < seg) ? bt[it + 32 + lane] : 0;
+                }
                 int page = __shfl_sync(0xffffffffu, btw, it & 31);
                 const bool page_ok = (page >= 0 && page < a.num_blocks);
                 if (!page_ok) { if (lane == 0) report(a.status, HOOK_ATTN_ERR_BOUNDS); page = 0; }
@@ -311,7 +299,8 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const Ker
         // ---- this warp's partial of unit (s, kvh) ----
         {
             const int h0 = 2 * tq, h1 = 2 * tq + 1;
-            float* part = a.ws + ((size_t)s * a.Hkv + kvh + W) * G * pstride;
+            float* part = reinterpret_cast<float*>(reinterpret_cast<char*>(a.ws) + decode_prefix_bytes(a.num_seqs)) +
+                          ((size_t)s * a.Hkv + kvh + W) * G * pstride;
             float* r0 = part + h0 * pstride;
             float* r1 = part + h1 * pstride;
 #pragma unroll
@@ -347,21 +336,239 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const Ker
     }
 }
 
+template <int HD, int NS>
+__global__ void __launch_bounds__(kDecWarps * 32) decode_splitk_kernel(const KernelArgs a, const HeadCfg hc)
+{
+    constexpr int ROWB = HD * 2;            // bytes per K/V row
+    constexpr int TILEB = kPage * ROWB;     // bytes per 16-key tile
+    constexpr int CPR = HD / 8;             // 16-byte chunks per row
+    constexpr int RPI = 32 / CPR;           // rows covered by one warp-wide copy instruction
+    constexpr int KS = HD / 16;             // k-steps of the score product / d-blocks of the output
+    constexpr int OSTR = HD + 4;            // padded row of the cross-warp reduction buffer
+
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ int sh_span[2 * kMaxSpans];
+    __shared__ float sh_m[kDecWarps][8];
+    __shared__ float sh_small[kDecWarps][8][2 + kMaxSpans];
+
+    const int s = blockIdx.z, kvh = blockIdx.y, c = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+    const int G = a.G;
+
+    const int L = a.seq_lens[s];
+    if (L <= 0 || L > a.max_blocks * kPage) return;   // reported and zero-filled by the merge kernel
+    const int start = c * a.chunk;
+    if (start >= L) return;
+    const int end = min(L, start + a.chunk);
+    const int ntiles = (end - start + kPage - 1) / kPage;
+
+    bool probe = false;
+    if constexpr (NS > 0) {
+        for (int i = 0; i < G; ++i) probe |= (hc.slot[kvh * G + i] >= 0);
+        if ((int)threadIdx.x < 2 * NS) {
+            const int j = threadIdx.x >> 1;
+            sh_span[threadIdx.x] = (probe && j < a.S) ? a.spans[((int64_t)s * a.S + j) * 2 + (threadIdx.x & 1)] : 0;
+        }
+    }
+    __syncthreads();
+
+    // B fragments of Q^T (k = d, n = head): head g of the group, zero for padding heads.
+    uint32_t qb[KS][2];
+    {
+        const __nv_bfloat16* qrow = a.q + ((int64_t)s * a.Hq + kvh * G + g) * HD;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            qb[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * tq) : 0u;
+            qb[ks][1] = (g < G) ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * tq) : 0u;
+        }
+    }
+
+    const uint32_t wbase = smem_u32(smem) + warp * (kDecStages * 2 * TILEB);
+    const int32_t* bt = a.block_table + (int64_t)s * a.max_blocks;
+    const int my_tiles = (ntiles > warp) ? (ntiles - warp + kDecWarps - 1) / kDecWarps : 0;
+
+    auto issue = [&](int it) {
+        if (it < my_tiles) {
+            const int key0 = start + (warp + it * kDecWarps) * kPage;
+            int page = bt[key0 / kPage];
+            bool page_ok = (page >= 0 && page < a.num_blocks);
+            if (!page_ok) { report(a.status, HOOK_ATTN_ERR_BOUNDS); page = 0; }
+            const uint32_t kdst = wbase + (it % kDecStages) * (2 * TILEB);
+            const uint32_t vdst = kdst + TILEB;
+            const int64_t base = (int64_t)page * a.bs + (int64_t)kvh * a.hs;
+#pragma unroll
+            for (int i = 0; i < kPage / RPI; ++i) {
+                const int r = i * RPI + lane / CPR;
+                const int cc = lane % CPR;
+                const bool ok = page_ok && (key0 + r < L);
+                const int64_t off = base + (int64_t)r * a.ts + cc * 8;
+                cp_async16(kdst + swz<ROWB>(r, cc), a.k + off, ok);
+                cp_async16(vdst + swz<ROWB>(r, cc), a.v + off, ok);
+            }
+        }
+        cp_async_commit();
+    };
+
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float o[KS][4];
+#pragma unroll
+    for (int i = 0; i < KS; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float sm[NS > 0 ? NS : 1][2];
+#pragma unroll
+    for (int j = 0; j < (NS > 0 ? NS : 1); ++j) sm[j][0] = sm[j][1] = 0.f;
+
+#pragma unroll
+    for (int i = 0; i < kDecStages - 1; ++i) issue(i);
+
+    for (int it = 0; it < my_tiles; ++it) {
+        issue(it + kDecStages - 1);
+        cp_async_wait<kDecStages - 1>();
+        __syncwarp();
+
+        const int key0 = start + (warp + it * kDecWarps) * kPage;
+        const uint32_t kt = wbase + (it % kDecStages) * (2 * TILEB);
+        const uint32_t vt = kt + TILEB;
+
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            uint32_t af[4];
+            ldmatrix_x4(af, kt + swz<ROWB>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)));
+            mma_bf16_16816(sc, af, qb[ks][0], qb[ks][1]);
+        }
+        const int t0 = key0 + g, t1 = t0 + 8;
+        const float x0 = (t0 < L) ? sc[0] * a.scale_log2 : -INFINITY;   // (key t0, head 2tq)
+        const float x1 = (t0 < L) ? sc[1] * a.scale_log2 : -INFINITY;   // (key t0, head 2tq+1)
+        const float x2 = (t1 < L) ? sc[2] * a.scale_log2 : -INFINITY;   // (key t1, head 2tq)
+        const float x3 = (t1 < L) ? sc[3] * a.scale_log2 : -INFINITY;   // (key t1, head 2tq+1)
+        float mx0 = fmaxf(x0, x2), mx1 = fmaxf(x1, x3);
+#pragma unroll
+        for (int d = 4; d <= 16; d <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, d));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, d));
+        }
+        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: key0 < L
+        const float c0 = fast_exp2(m0 - mn0), c1 = fast_exp2(m1 - mn1);
+        m0 = mn0; m1 = mn1;
+        const float p0 = fast_exp2(x0 - mn0), p1 = fast_exp2(x1 - mn1);
+        const float p2 = fast_exp2(x2 - mn0), p3 = fast_exp2(x3 - mn1);
+        l0 = l0 * c0 + (p0 + p2);
+        l1 = l1 * c1 + (p1 + p3);
+#pragma unroll
+        for (int i = 0; i < KS; ++i) { o[i][0] *= c0; o[i][1] *= c1; o[i][2] *= c0; o[i][3] *= c1; }
+
+        if (NS > 0 && probe) {
+#pragma unroll
+            for (int j = 0; j < NS; ++j) {
+                const int sa = sh_span[2 * j], sb = sh_span[2 * j + 1];
+                float add0 = 0.f, add1 = 0.f;
+                if (sb > key0 && sa < key0 + kPage) {
+                    const bool in0 = (t0 >= sa) && (t0 < sb), in1 = (t1 >= sa) && (t1 < sb);
+                    add0 = (in0 ? p0 : 0.f) + (in1 ? p2 : 0.f);
+                    add1 = (in0 ? p1 : 0.f) + (in1 ? p3 : 0.f);
+                }
+                sm[j][0] = sm[j][0] * c0 + add0;
+                sm[j][1] = sm[j][1] * c1 + add1;
+            }
+        }
+
+        // P^T as the B operand (k = key, n = head): transpose the two 8x8 blocks across lanes.
+        const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
+        const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
+#pragma unroll
+        for (int i = 0; i < KS; ++i) {
+            uint32_t af[4];
+            ldmatrix_x4_trans(af, vt + swz<ROWB>((lane & 7) + (lane >> 4) * 8, 2 * i + ((lane >> 3) & 1)));
+            mma_bf16_16816(o[i], af, pb0, pb1);
+        }
+        __syncwarp();
+    }
+    cp_async_wait<0>();
+
+    // per-thread partial sums -> per-warp sums (lanes with the same tq hold the same heads)
+#pragma unroll
+    for (int d = 4; d <= 16; d <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, d);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, d);
+        if (NS > 0) {
+#pragma unroll
+            for (int j = 0; j < NS; ++j) {
+                sm[j][0] += __shfl_xor_sync(0xffffffffu, sm[j][0], d);
+                sm[j][1] += __shfl_xor_sync(0xffffffffu, sm[j][1], d);
+            }
+        }
+    }
+
+    // ---- merge the four warps ----
+    if (g == 0) { sh_m[warp][2 * tq] = m0; sh_m[warp][2 * tq + 1] = m1; }
+    __syncthreads();   // also: every warp has drained its pipeline, the stage buffers are free
+    float M0 = sh_m[0][2 * tq], M1 = sh_m[0][2 * tq + 1];
+#pragma unroll
+    for (int w = 1; w < kDecWarps; ++w) { M0 = fmaxf(M0, sh_m[w][2 * tq]); M1 = fmaxf(M1, sh_m[w][2 * tq + 1]); }
+    const float f0 = fast_exp2(m0 - M0), f1 = fast_exp2(m1 - M1);   // warp without tiles: m = -inf -> 0
+
+    float* red = reinterpret_cast<float*>(smem);   // [warps][8 heads][OSTR]
+#pragma unroll
+    for (int i = 0; i < KS; ++i) {
+        float* r0 = red + (warp * 8 + 2 * tq) * OSTR;
+        r0[16 * i + g] = o[i][0] * f0;
+        r0[OSTR + 16 * i + g] = o[i][1] * f1;
+        r0[16 * i + 8 + g] = o[i][2] * f0;
+        r0[OSTR + 16 * i + 8 + g] = o[i][3] * f1;
+    }
+    if (g == 0) {
+        sh_small[warp][2 * tq][0] = M0;
+        sh_small[warp][2 * tq + 1][0] = M1;
+        sh_small[warp][2 * tq][1] = l0 * f0;
+        sh_small[warp][2 * tq + 1][1] = l1 * f1;
+        if (NS > 0) {
+#pragma unroll
+            for (int j = 0; j < NS; ++j) {
+                sh_small[warp][2 * tq][2 + j] = sm[j][0] * f0;
+                sh_small[warp][2 * tq + 1][2 + j] = sm[j][1] * f1;
+            }
+        }
+    }
+    __syncthreads();
+
+    const size_t pstride = decode_partial_stride(HD);
+    float* part = a.ws + (((size_t)s * a.Hkv + kvh) * a.max_chunks + c) * G * pstride;
+    for (int idx = threadIdx.x; idx < G * HD; idx += kDecWarps * 32) {
+        const int h = idx / HD, d = idx % HD;
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kDecWarps; ++w) acc += red[(w * 8 + h) * OSTR + d];
+        part[h * pstride + d] = acc;
+    }
+    for (int idx = threadIdx.x; idx < G * (2 + NS); idx += kDecWarps * 32) {
+        const int h = idx / (2 + NS), e = idx % (2 + NS);
+        float val;
+        if (e == 0) {
+            val = sh_small[0][h][0];
+        } else {
+            val = 0.f;
+#pragma unroll
+            for (int w = 0; w < kDecWarps; ++w) val += sh_small[w][h][e];
+        }
+        part[h * pstride + HD + e] = val;
+    }
+}
+
 constexpr int kMergeMaxWarps = 16;   // warps of the merge kernel when a unit may have many partials (4 otherwise)
 
-// One CTA per (query head, sequence).  From the sequence lengths it recomputes which worker warps
-// of the streaming kernel covered the unit (the same arithmetic as there), then warp w folds the
-// partials w, w + nwarps, ... with an online rescale (all loads of a partial are independent of the
-// previous one's arithmetic, so several are in flight); the warps are then combined in warp order
-// by the first 128 threads.  The order of every floating-point sum is fixed by (partial, warp)
-// indices only: run-to-run bit-identical.
-template <int HD>
+// One CTA per (query head, sequence).  It finds the unit's partials -- the chunks of the sequence, or
+// the worker warps of the streaming kernel that covered the unit (the same arithmetic as there, from
+// the page-count prefix that kernel left) -- then warp w folds the partials w, w + nwarps, ... with an
+// online rescale (all loads of a partial are independent of the previous one's arithmetic, so several
+// are in flight); the warps are then combined in warp order by the first 128 threads.  The order of
+// every floating-point sum is fixed by (partial, warp) indices only: run-to-run bit-identical.
+template <int HD, bool STREAM>
 __global__ void __launch_bounds__(kMergeMaxWarps * 32) decode_merge_kernel(const KernelArgs a, const HeadCfg hc)
 {
     constexpr int EPL = HD / 32;                       // output elements per lane
     __shared__ float sh_acc[kMergeMaxWarps][HD];
     __shared__ float sh_small[kMergeMaxWarps][2 + kMaxSpans];   // M, l, s[0..7]
-    __shared__ int sh_cnt[kMergeMaxWarps][2];
 
     const int h = blockIdx.x, s = blockIdx.y;
     const int G = a.G, kvh = h / G, gi = h % G;
@@ -371,42 +578,33 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) decode_merge_kernel(const
     const int slot = hc.slot[h];
     float* mrow = (slot >= 0 && a.S > 0) ? a.mass + ((int64_t)s * a.P + slot) * a.S : nullptr;
 
-    // pages before this sequence and in total: inputs of the call only, so this runs while the
-    // streaming kernel is still at work
-    int before = 0, total = 0;
-    for (int i = threadIdx.x; i < a.num_seqs; i += blockDim.x) {
-        const int pgs = decode_pages(a.seq_lens[i], a.max_blocks);
-        total += pgs;
-        if (i < s) before += pgs;
-    }
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) {
-        before += __shfl_xor_sync(0xffffffffu, before, d);
-        total += __shfl_xor_sync(0xffffffffu, total, d);
-    }
-    if (lane == 0) { sh_cnt[warp][0] = before; sh_cnt[warp][1] = total; }
-    __syncthreads();
-    before = 0; total = 0;
-    for (int w = 0; w < nwarps; ++w) { before += sh_cnt[w][0]; total += sh_cnt[w][1]; }
-    const int L = a.seq_lens[s];
-    const int np = decode_pages(L, a.max_blocks);
-
-    // the partials are written by the streaming kernel launched just before on the same stream
+    // the partials are written by the kernel launched just before on the same stream
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
+    const int L = a.seq_lens[s];
+    const int np = decode_pages(L, a.max_blocks);
     if (np == 0) {
         if (threadIdx.x == 0) report(a.status, L <= 0 ? HOOK_ATTN_ERR_INVALID_ARG : HOOK_ATTN_ERR_BOUNDS);
         if ((int)threadIdx.x < HD) orow[threadIdx.x] = __float2bfloat16(0.f);
         if (mrow && (int)threadIdx.x < a.S) mrow[threadIdx.x] = 0.f;
         return;
     }
-    const long long share = decode_share((long long)total * a.Hkv, a.workers);
-    const long long f0 = (long long)before * a.Hkv + (long long)kvh * np;   // the unit's pages in the flat list
-    const int w_first = (int)(f0 / share), w_last = (int)((f0 + np - 1) / share);
-    const int nchunks = w_last - w_first + 1;
     const size_t pstride = decode_partial_stride(HD);
-    const float* part = a.ws + (((size_t)s * a.Hkv + kvh + w_first) * G + gi) * pstride;
     const size_t cstride = (size_t)G * pstride;
+    int nchunks;
+    const float* part;
+    if (STREAM) {
+        const int* prefix = reinterpret_cast<const int*>(a.ws);
+        const long long share = decode_share((long long)prefix[a.num_seqs] * a.Hkv);
+        const long long f0 = (long long)prefix[s] * a.Hkv + (long long)kvh * np;   // the unit's pages in the flat list
+        const int w_first = (int)(f0 / share), w_last = (int)((f0 + np - 1) / share);
+        nchunks = w_last - w_first + 1;
+        part = reinterpret_cast<const float*>(reinterpret_cast<const char*>(a.ws) + decode_prefix_bytes(a.num_seqs)) +
+               (((size_t)s * a.Hkv + kvh + w_first) * G + gi) * pstride;
+    } else {
+        nchunks = (L + a.chunk - 1) / a.chunk;
+        part = a.ws + ((((size_t)s * a.Hkv + kvh) * a.max_chunks) * G + gi) * pstride;
+    }
     const bool want_mass = mrow != nullptr;
 
     float M = -INFINITY, lsum = 0.f, sacc = 0.f, acc[EPL];
@@ -457,21 +655,51 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) decode_merge_kernel(const
 }
 
 // ------------------------------------------------------------------------------------------
-template <int HD, int NS>
-static cudaError_t launch_decode_t(const KernelArgs& a, const HeadCfg& hc, cudaStream_t st)
+// How a call is cut into pieces, from host-known bounds only (the lengths live on the device).
+struct DecodePlan {
+    bool stream;      // streaming kernel (few units) or fixed chunks
+    int chunk;        // fixed chunks: keys per chunk, the largest power of two in 256..2048 that still
+    int max_chunks;   //   leaves at least eight CTAs per SM in the grid; chunks per sequence
+};
+
+static DecodePlan decode_plan(int num_seqs, int Hkv, int max_blocks)
 {
-    decode_stream_kernel<HD, NS><<<a.workers / kDecWarps, kDecWarps * 32, decode_smem_bytes<HD>(), st>>>(a, hc);
+    DecodePlan p = {};
+    p.stream = (long)num_seqs * Hkv < kDecCtas;
+    const long max_keys = (long)max_blocks * kPage;
+    p.chunk = 2048;
+    while (p.chunk > 256) {
+        const long ctas = (long)num_seqs * Hkv * ((max_keys + p.chunk - 1) / p.chunk);
+        if (ctas >= 8L * 148) break;
+        p.chunk >>= 1;
+    }
+    p.max_chunks = (int)((max_keys + p.chunk - 1) / p.chunk);
+    if (p.max_chunks < 1) p.max_chunks = 1;
+    return p;
+}
+
+template <int HD, int NS>
+static cudaError_t launch_decode_t(KernelArgs a, const HeadCfg& hc, cudaStream_t st)
+{
+    const DecodePlan plan = decode_plan(a.num_seqs, a.Hkv, a.max_blocks);
+    a.chunk = plan.chunk;
+    a.max_chunks = plan.max_chunks;
+    long parts;   // partials per unit, to size the merge block
+    if (plan.stream) {
+        decode_stream_kernel<HD, NS><<<kDecCtas, kDecWarps * 32, decode_smem_bytes<HD>(), st>>>(a, hc);
+        const long est_share = ((long)a.num_seqs * a.Hkv * a.max_blocks / 2 + kDecWorkers - 1) / kDecWorkers;
+        parts = a.max_blocks / (est_share > 0 ? est_share : 1) + 2;
+    } else {
+        decode_splitk_kernel<HD, NS><<<dim3(plan.max_chunks, a.Hkv, a.num_seqs), kDecWarps * 32, decode_smem_bytes<HD>(), st>>>(a, hc);
+        parts = plan.max_chunks;
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    // The merge is launched with programmatic stream serialization: its CTAs may become resident
-    // while the streaming kernel runs, size up their unit from the sequence lengths, and wait
-    // (griddepcontrol.wait) until that kernel has finished and its writes are visible.
-    // Expected partials per unit when lengths average half the table: pick the wide block for many.
-    const long est_share = ((long)a.num_seqs * a.Hkv * a.max_blocks / 2 + a.workers - 1) / a.workers;
-    const long est_parts = a.max_blocks / (est_share > 0 ? est_share : 1) + 2;
+    // The merge is launched with programmatic stream serialization: its launch overlaps the drain of
+    // the first kernel, and it waits (griddepcontrol.wait) until that kernel's writes are visible.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.Hq, a.num_seqs);
-    cfg.blockDim = dim3((est_parts > 8 ? kMergeMaxWarps : 4) * 32);
+    cfg.blockDim = dim3((parts > 8 ? kMergeMaxWarps : 4) * 32);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -479,17 +707,21 @@ static cudaError_t launch_decode_t(const KernelArgs& a, const HeadCfg& hc, cudaS
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_merge_kernel<HD>, a, hc);
+    return plan.stream ? cudaLaunchKernelEx(&cfg, decode_merge_kernel<HD, true>, a, hc)
+                       : cudaLaunchKernelEx(&cfg, decode_merge_kernel<HD, false>, a, hc);
 }
 
 template <int HD, int NS>
 static cudaError_t configure_one()
 {
+    cudaError_t e = cudaFuncSetAttribute(decode_splitk_kernel<HD, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         decode_smem_bytes<HD>());
+    if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(decode_stream_kernel<HD, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 decode_smem_bytes<HD>());
 }
 
-// Opt in to the dynamic shared memory the split-K kernels use (per device; called with the
+// Opt in to the dynamic shared memory the first-stage kernels use (per device; called with the
 // device current when a handle is created).
 cudaError_t configure_decode()
 {
@@ -501,17 +733,14 @@ cudaError_t configure_decode()
     return cudaSuccess;
 }
 
-// Worker warps of the streaming kernel for a call of these bounds.
-int decode_workers(int num_seqs, int Hkv, int head_dim, int max_blocks)
-{
-    return decode_rounds(num_seqs, Hkv, head_dim, max_blocks) * kDecCtas * kDecWarps;
-}
-
-// One partial per (unit, worker warp) pair that meets; the slot `unit + warp` is below units + workers.
+// Fixed chunks: one partial per (unit, chunk).  Streaming: the page-count prefix, then one partial
+// per (unit, worker warp) pair that meets; the slot `unit + warp` is below units + workers.
 size_t decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim, int max_blocks)
 {
-    return ((size_t)num_seqs * Hkv + decode_workers(num_seqs, Hkv, head_dim, max_blocks)) * G *
-           decode_partial_stride(head_dim) * sizeof(float);
+    const DecodePlan plan = decode_plan(num_seqs, Hkv, max_blocks);
+    const size_t per_part = (size_t)G * decode_partial_stride(head_dim) * sizeof(float);
+    if (plan.stream) return decode_prefix_bytes(num_seqs) + ((size_t)num_seqs * Hkv + kDecWorkers) * per_part;
+    return (size_t)num_seqs * Hkv * plan.max_chunks * per_part;
 }
 
 cudaError_t launch_decode(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st)

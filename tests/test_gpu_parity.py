@@ -128,28 +128,31 @@ def test_decode_shapes_and_ragged_lengths(eng, Hq, Hkv, D):
     check(eng, case)
 
 
-def test_decode_page_shares_many_and_skewed_sequences(eng):
-    """The decode kernel deals the pages of all sequences out to its workers in equal shares.  Here: more
-    sequences than one window of its page-count scan (1024), lengths from one key to hundreds of pages, two
-    long sequences that many workers share, workers whose share crosses dozens of short sequences, and
-    then the same batch with empty sequences in the middle (reported, zero-filled, the rest untouched)."""
-    g = inputs._gen(4242)
-    lens = torch.randint(1, 40, (1300,), generator=g).tolist()
-    lens[7], lens[1100] = 9000, 5000
+@pytest.mark.parametrize("num_seqs,holes", [(140, (3, 70, 139)), (1300, (3, 1023, 1024, 1200))])
+def test_decode_skewed_batches_in_both_ways_of_cutting(eng, num_seqs, holes):
+    """Decode cuts a batch in one of two ways.  With fewer than 296 (sequence, KV head) units the pages
+    of all sequences are dealt out to the worker warps in equal shares: here lengths from one key to
+    hundreds of pages, two long sequences that many workers share, workers whose share crosses dozens
+    of short sequences.  With more units each sequence is cut into fixed chunks: here more than a
+    thousand sequences.  Then the same batch with empty sequences in the middle (reported, zero-filled,
+    the rest untouched)."""
+    g = inputs._gen(4242 + num_seqs)
+    lens = torch.randint(1, 40, (num_seqs,), generator=g).tolist()
+    lens[7], lens[num_seqs - 30] = 9000, 5000
     alpha = torch.zeros(4)
     alpha[1] = -0.6
-    case = inputs.make_case("dec_many", is_decode=True, seq_lens=lens, q_lens=[1] * len(lens), num_q_heads=4,
+    case = inputs.make_case("dec_skewed", is_decode=True, seq_lens=lens, q_lens=[1] * len(lens), num_q_heads=4,
                             num_kv_heads=2, head_dim=64, seed=4243, num_spans=2,
                             head_mask=torch.tensor([1, 0, 1, 1], dtype=torch.uint8), alpha=alpha, steer=True,
                             probe_rows=inputs.PROBE_ROWS_LAST, poison=True)
     check(eng, case)
     out0, mass0, _ = run_gpu(eng, case)
-    holes = list(lens)
-    for i in (3, 1023, 1024, 1200):
-        holes[i] = 0
-    out1, mass1, st = run_gpu(eng, inputs.with_seq_lens(case, holes))
+    shorter = list(lens)
+    for i in holes:
+        shorter[i] = 0
+    out1, mass1, st = run_gpu(eng, inputs.with_seq_lens(case, shorter))
     assert st == binding.HOOK_ATTN_ERR_INVALID_ARG
-    keep = torch.tensor([i not in (3, 1023, 1024, 1200) for i in range(len(lens))], device=out0.device)
+    keep = torch.tensor([i not in holes for i in range(len(lens))], device=out0.device)
     assert torch.all(out1[~keep] == 0) and torch.all(mass1[~keep] == 0)
     assert (out1[keep].float() - out0[keep].float()).abs().max().item() <= TOL_OUT
     assert (mass1[keep] - mass0[keep]).abs().max().item() <= TOL_MASS
