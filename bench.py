@@ -55,7 +55,8 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu captures
 # summarised under profiles/ (None where no capture of the current kernel exists).
 DRAM_TRAFFIC = {
-    "cfg2_decode": 625.15e6 + 6.59e6,     # profiles/decode_splitk_kernel__cfg2_decode.md
+    "cfg2_decode": 625.11e6 + 6.70e6,     # profiles/decode_splitk_kernel__cfg2_decode.md
+    "cfg5_decode": 538.10e6 + 4.26e6,     # profiles/decode_stream_kernel__cfg5_decode.md
     "cfg3_prefill_small": 50.41e6 + 3.83e6,   # profiles/prefill_tc_kernel__cfg3_prefill_small.md
 }
 
@@ -634,7 +635,8 @@ def main():
                        "replicas": world, "kv_cache": "resident in HBM (state, not a per-step input)"},
             "roofline": {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
                          "traffic": DRAM_TRAFFIC.get(args.workload), "peak_source": f"of {peaks['source']}",
-                         "kernel": "decode_splitk_kernel (+ decode_merge_kernel; duration = whole step, conservative)"
+                         "kernel": (("decode_stream_kernel" if case.num_seqs * case.num_kv_heads < 296 else "decode_splitk_kernel")
+                                    + " (+ decode_merge_kernel; duration = whole step, conservative)")
                          if case.is_decode else "prefill_tc_kernel (one launch per step)",
                          "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
                          "frac_of_datasheet": achieved / (8000.0 if bound == "hbm" else 2250.0)},
