@@ -48,19 +48,6 @@ constexpr int kStages = 2;
 constexpr int kSmemBytes = 2 * kTileBytes + 2 * kStages * kTileBytes + 1024;   // Q(A,B) + K,V stages + alignment slack
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.0f;       // log2 units
-// Of every eight pairs of probabilities, this many are computed with a polynomial on the FMA pipe
-// instead of the special-function unit (which gives 16 results per clock and SM and would otherwise
-// set the pace of the softmax).
-#ifndef HOOK_TC_POLY_PER8
-#define HOOK_TC_POLY_PER8 0
-#endif
-constexpr int kPolyPer8 = HOOK_TC_POLY_PER8;
-// The probabilities of a tile are handed to the MMA thread in two halves of 64 keys, so that P V of
-// the first half runs while the second half is still being exponentiated.
-#ifndef HOOK_TC_SPLIT_P
-#define HOOK_TC_SPLIT_P 0
-#endif
-constexpr bool kSplitP = HOOK_TC_SPLIT_P != 0;
 constexpr int kMaskTiles = 1024;                // key tiles with a precomputed span classification
 
 // Which spans does key tile [k0, k0 + 128) touch?  Low byte: spans that contain the whole tile;
@@ -212,25 +199,6 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-// 2^x for a pair of arguments x <= 8 on the FMA pipe: x = n + f with n = round(x) (magic-number
-// add), 2^f on [-1/2, 1/2] from a degree-4 polynomial (relative error 3e-6), 2^n added into the
-// exponent field.  Arguments below -126 (masked keys are -inf) give a value below 1e-37.
-__device__ __forceinline__ float2 poly_exp2(float2 x)
-{
-    const float kMagic = 12582912.f;   // 1.5 * 2^23: the sum's low mantissa bits are round(x)
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    const float2 t = __fadd2_rn(x, make_float2(kMagic, kMagic));
-    const float2 n = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
-    const float2 f = __ffma2_rn(n, make_float2(-1.f, -1.f), x);
-    float2 p = make_float2(0.00957401655614376f, 0.00957401655614376f);
-    p = __ffma2_rn(p, f, make_float2(0.055918190628290176f, 0.055918190628290176f));
-    p = __ffma2_rn(p, f, make_float2(0.2402464896440506f, 0.2402464896440506f));
-    p = __ffma2_rn(p, f, make_float2(0.6931217312812805f, 0.6931217312812805f));
-    p = __ffma2_rn(p, f, make_float2(0.9999992847442627f, 0.9999992847442627f));
-    return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),
-                       __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
-}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
@@ -254,7 +222,6 @@ struct Barriers {
     uint64_t q_full[2];
     uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
     uint64_t s_full[2], p_full[2], o_full[2];
-    uint64_t p_half[2];       // the first 64 keys' probabilities of a tile are in tensor memory
     uint64_t v_tail;          // the producer has zeroed the value rows past the end of the sequence
     uint32_t tmem_base;
     int abort_flag;
@@ -318,12 +285,13 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
     const uint32_t sV = sK + kStages * kTileBytes;
 
     // ---- set-up: barriers, spans, tensor memory ----
-    if (threadIdx.x == 0) {
+    // The producer warp initialises the barriers and at once starts the loads of Q and of the first
+    // K/V tile, so that their latency runs under the rest of the set-up.
+    if (warp == kProducerWarp && lane == 0) {
         for (int x = 0; x < 2; ++x) {
             mbar_init(smem_u32(&bars.q_full[x]), 1);
             mbar_init(smem_u32(&bars.s_full[x]), 1);
             mbar_init(smem_u32(&bars.p_full[x]), 128);
-            mbar_init(smem_u32(&bars.p_half[x]), 128);
             mbar_init(smem_u32(&bars.o_full[x]), 1);
         }
         for (int i = 0; i < kStages; ++i) {
@@ -335,6 +303,48 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
         mbar_init(smem_u32(&bars.v_tail), 1);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    bool ok = true;   // false once a bounded wait ran out
+    const int32_t* bt = a.block_table + (int64_t)s * a.max_blocks;
+    // producer: the loads of key tile j (K then V), one TMA box per (page, 64-wide half of the head)
+    auto produce = [&](int j) {
+        const int st = j & 1;
+        const uint32_t ph = (j >> 1) & 1;
+        const int pages = min(kBN / kPage, (L - j * kBN + kPage - 1) / kPage);   // pages that hold keys < L
+        int blk = 0;
+        const int pg = lane >> 1, half = lane & 1;
+        if (lane < 16 && pg < pages) {
+            blk = bt[j * (kBN / kPage) + pg];
+            if (blk < 0 || blk >= a.num_blocks) { report(a.status, HOOK_ATTN_ERR_BOUNDS); blk = 0; }
+        }
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv) {
+            const uint32_t full = smem_u32(kv ? &bars.v_full[st] : &bars.k_full[st]);
+            const uint32_t empty = smem_u32(kv ? &bars.v_empty[st] : &bars.k_empty[st]);
+            ok = __all_sync(0xffffffffu, mbar_wait(empty, ph ^ 1u));
+            if (!ok) break;
+            if (lane == 0) mbar_expect_tx(full, (uint32_t)pages * 2u * (kPage * 128u));
+            __syncwarp();
+            if (lane < 16 && pg < pages) {
+                const uint32_t dst = (kv ? sV : sK) + st * kTileBytes + half * kHalfBytes + pg * (kPage * 128);
+                tma_load_4d(dst, kv ? &map_v : &map_k, full, half * 64, kvh, 0, blk);
+            }
+        }
+    };
+    if (warp == kProducerWarp) {
+        __syncwarp();
+        if (lane == 0) {
+#pragma unroll
+            for (int x = 0; x < 2; ++x) {
+                if (ntiles[x] > 0) {
+                    const uint32_t bar = smem_u32(&bars.q_full[x]);
+                    mbar_expect_tx(bar, kTileBytes);
+                    tma_load_3d(sQ[x], &map_q, bar, 0, h, (int)(grow_seq + row0[x]));
+                    tma_load_3d(sQ[x] + kHalfBytes, &map_q, bar, 64, h, (int)(grow_seq + row0[x]));
+                }
+            }
+        }
+        if (nmax > 0) produce(0);
     }
     if (NS > 0 && (int)threadIdx.x < 2 * NS) {
         const int j = threadIdx.x >> 1;
@@ -353,7 +363,6 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = bars.tmem_base;
-    bool ok = true;   // false once a bounded wait ran out
 
     // Register split between the warpgroups: the softmax threads keep a whole 128-wide score row in
     // registers, the producer/MMA warpgroup needs few.  Launched with 168 per thread (384 x 168 =
@@ -366,42 +375,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
     }
     if (warp == kProducerWarp) {
         // ================================ producer ================================
-        const int32_t* bt = a.block_table + (int64_t)s * a.max_blocks;
-        if (lane == 0) {
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                if (ntiles[x] > 0) {
-                    const uint32_t bar = smem_u32(&bars.q_full[x]);
-                    mbar_expect_tx(bar, kTileBytes);
-                    tma_load_3d(sQ[x], &map_q, bar, 0, h, (int)(grow_seq + row0[x]));
-                    tma_load_3d(sQ[x] + kHalfBytes, &map_q, bar, 64, h, (int)(grow_seq + row0[x]));
-                }
-            }
-        }
-        for (int j = 0; j < nmax && ok; ++j) {
-            const int st = j & 1;
-            const uint32_t ph = (j >> 1) & 1;
-            const int pages = min(kBN / kPage, (L - j * kBN + kPage - 1) / kPage);   // pages that hold keys < L
-            int blk = 0;
-            const int pg = lane >> 1, half = lane & 1;
-            if (lane < 16 && pg < pages) {
-                blk = bt[j * (kBN / kPage) + pg];
-                if (blk < 0 || blk >= a.num_blocks) { report(a.status, HOOK_ATTN_ERR_BOUNDS); blk = 0; }
-            }
-#pragma unroll
-            for (int kv = 0; kv < 2; ++kv) {
-                const uint32_t full = smem_u32(kv ? &bars.v_full[st] : &bars.k_full[st]);
-                const uint32_t empty = smem_u32(kv ? &bars.v_empty[st] : &bars.k_empty[st]);
-                ok = __all_sync(0xffffffffu, mbar_wait(empty, ph ^ 1u));
-                if (!ok) break;
-                if (lane == 0) mbar_expect_tx(full, (uint32_t)pages * 2u * (kPage * 128u));
-                __syncwarp();
-                if (lane < 16 && pg < pages) {
-                    const uint32_t dst = (kv ? sV : sK) + st * kTileBytes + half * kHalfBytes + pg * (kPage * 128);
-                    tma_load_4d(dst, kv ? &map_v : &map_k, full, half * 64, kvh, 0, blk);
-                }
-            }
-        }
+        for (int j = 1; j < nmax && ok; ++j) produce(j);
         if (ok && nmax > 0 && nmax * kBN > L) {
             // value rows at keys >= L (page tails, pages that were never loaded) must not reach the
             // tensor cores: 0 * NaN would poison the accumulator.  Zero them in shared memory once the
@@ -439,10 +413,10 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             }
             tc_commit(smem_u32(&bars.s_full[x]));
         };
-        auto issue_pv = [&](int x, int j, int ks0, int ks1) {
+        auto issue_pv = [&](int x, int j) {
             const uint64_t dv = (j & 1) ? dV[1] : dV[0];
 #pragma unroll
-            for (int ks = ks0; ks < ks1; ++ks)
+            for (int ks = 0; ks < kBN / 16; ++ks)
                 tc_mma_ts(tO[x], tS[x] + ks * 8, desc_advance(dv, (ks * 16 * 128) >> 4), idesc_pv, (ks > 0) || (j > 0));
         };
         if (lane == 0) {
@@ -464,16 +438,10 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
 #pragma unroll
                 for (int x = 0; x < 2; ++x) {
                     if (ok && j < ntiles[x]) {
-                        if (kSplitP) {
-                            ok = mbar_wait(smem_u32(&bars.p_half[x]), j & 1);
-                            if (!ok) break;
-                            tc_fence_after();
-                            issue_pv(x, j, 0, kBN / 32);
-                        }
                         ok = mbar_wait(smem_u32(&bars.p_full[x]), j & 1);
                         if (!ok) break;
                         tc_fence_after();
-                        issue_pv(x, j, kSplitP ? kBN / 32 : 0, kBN / 16);
+                        issue_pv(x, j);
                         if (j + 1 < ntiles[x]) issue_qk(x, j + 1);
                         else tc_commit(smem_u32(&bars.o_full[x]));
                     }
@@ -571,18 +539,13 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
                     for (int i = 0; i < 16; ++i) {
                         const int e = 32 * c + 2 * i;
                         const float2 xx = __ffma2_rn(make_float2(sc[e], sc[e + 1]), sl2v, nmv);
-                        const float2 pp = ((i & 7) < kPolyPer8) ? poly_exp2(xx) : make_float2(fast_exp2(xx.x), fast_exp2(xx.y));
+                        const float2 pp = make_float2(fast_exp2(xx.x), fast_exp2(xx.y));
                         sc[e] = pp.x;
                         sc[e + 1] = pp.y;
                         rs2[i & 1] = __fadd2_rn(rs2[i & 1], pp);
                         pk[i] = pack_bf16(pp.x, pp.y);
                     }
                     tc_st16(tS + 16 * c, pk);
-                    if (kSplitP && c == 1) {
-                        tc_wait_st();
-                        tc_fence_before();
-                        mbar_arrive(smem_u32(&bars.p_half[x]));
-                    }
                 }
                 const float rs = (rs2[0].x + rs2[0].y) + (rs2[1].x + rs2[1].y);
                 l += rs;
@@ -626,30 +589,51 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
 
             // ---- epilogue: normalise, steer, round once, store ----
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_full[x]), 0));
+            const float inv = 1.f / l;
+            const bool live = row < rows[x];
+            const uint32_t stage = sQ[x];
             if (ok) {
                 tc_fence_after();
-                const float inv = 1.f / l;
                 const float al = hc.alpha[h];
                 const float* sv = a.steer + (int64_t)h * kHD;
-                const bool live = row < rows[x];
-                __nv_bfloat16* orow = a.out + ((grow_seq + row0[x] + row) * a.Hq + h) * kHD;
+                // A thread holds one output row; stored from here, a warp would write 32 rows with 16
+                // bytes each per instruction.  The tile goes through the shared memory of Q_x instead
+                // (free: every MMA of this tile has completed), 16-byte chunks XOR-ed with the row so
+                // that neither side has bank conflicts, and leaves it two whole rows per instruction.
                 float v[32];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     tc_ld32(tO + 32 * c, v);
                     tc_wait_ld_dep(v);
-                    if (live) {
 #pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) {
-                            uint32_t w[4];
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint32_t w[4];
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const int d = 32 * c + 8 * q4 + 2 * i;
-                                float y0 = v[8 * q4 + 2 * i] * inv, y1 = v[8 * q4 + 2 * i + 1] * inv;
-                                if (al != 0.f) { y0 = fmaf(al, sv[d], y0); y1 = fmaf(al, sv[d + 1], y1); }
-                                w[i] = pack_bf16(y0, y1);
-                            }
-                            *reinterpret_cast<uint4*>(orow + 32 * c + 8 * q4) = make_uint4(w[0], w[1], w[2], w[3]);
+                        for (int i = 0; i < 4; ++i) {
+                            const int d = 32 * c + 8 * q4 + 2 * i;
+                            float y0 = v[8 * q4 + 2 * i] * inv, y1 = v[8 * q4 + 2 * i + 1] * inv;
+                            if (al != 0.f) { y0 = fmaf(al, sv[d], y0); y1 = fmaf(al, sv[d + 1], y1); }
+                            w[i] = pack_bf16(y0, y1);
+                        }
+                        const uint32_t addr = stage + row * 256 + (((4 * c + q4) ^ (row & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+                    }
+                }
+            }
+            // all four warps of the tile meet here, also one whose waits ran out (it reported that)
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + x) : "memory");
+            if (ok) {
+                {
+                    const int t128 = threadIdx.x & 127;
+                    __nv_bfloat16* otile = a.out + ((grow_seq + row0[x]) * a.Hq + h) * kHD;
+#pragma unroll 4
+                    for (int it = 0; it < 16; ++it) {
+                        const int idx = it * 128 + t128, r = idx >> 4, c = idx & 15;
+                        if (r < rows[x]) {
+                            uint4 val;
+                            const uint32_t addr = stage + r * 256 + ((c ^ (r & 7)) << 4);
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(val.x), "=r"(val.y), "=r"(val.z), "=r"(val.w) : "r"(addr));
+                            *reinterpret_cast<uint4*>(otile + (int64_t)r * a.Hq * kHD + c * 8) = val;
                         }
                     }
                 }
