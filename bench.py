@@ -57,7 +57,7 @@ WORKLOADS = {
 DRAM_TRAFFIC = {
     "cfg2_decode": 625.11e6 + 6.70e6,     # profiles/decode_splitk_kernel__cfg2_decode.md
     "cfg5_decode": 538.10e6 + 4.26e6,     # profiles/decode_stream_kernel__cfg5_decode.md
-    "cfg3_prefill_small": 50.41e6 + 3.83e6,   # profiles/prefill_tc_kernel__cfg3_prefill_small.md
+    "cfg3_prefill_small": 50.42e6 + 4.53e6,   # profiles/prefill_tc_kernel__cfg3_prefill_small.md
 }
 
 
