@@ -61,6 +61,82 @@ __device__ __forceinline__ long long decode_share(long long flat_total)
 __host__ __device__ inline size_t decode_prefix_bytes(int num_seqs) { return (((size_t)num_seqs + 1) * 4 + 255) & ~(size_t)255; }
 
 
+// One 16-key page of a unit: scores of the page against the G query heads, online softmax, span
+// accumulators, P V.  Thread layout of the warp-level MMA: lane = 4 g + tq holds keys g and g + 8 of the
+// page for the heads 2 tq and 2 tq + 1.  The softmax keeps a reference maximum per head that is only
+// raised when a score exceeds it by more than 2^8: probabilities, running sum, span accumulators and the
+// output all live in that frame (the reference cancels in o / l and s_j / l, so the result is exact),
+// and the common page needs neither the shuffles of a row maximum nor a rescale of the accumulators.
+constexpr float kDecRaise = 8.0f;   // log2 units
+
+template <int HD, int NS>
+__device__ __forceinline__ void decode_page(uint32_t kt, uint32_t vt, int key0, int L, float scale_log2, bool probe,
+                                            const int* span, const uint32_t (&qb)[HD / 16][2], float& m0, float& m1,
+                                            float& l0, float& l1, float (&o)[HD / 16][4], float (&sm)[NS > 0 ? NS : 1][2])
+{
+    constexpr int ROWB = HD * 2;
+    constexpr int KS = HD / 16;
+    const int lane = threadIdx.x & 31, g = lane >> 2;
+    float sca[4] = {0.f, 0.f, 0.f, 0.f}, scb[4] = {0.f, 0.f, 0.f, 0.f};   // two chains: half the dependent depth
+#pragma unroll
+    for (int ks = 0; ks < KS; ks += 2) {
+        uint32_t af[4], bf[4];
+        ldmatrix_x4(af, kt + swz<ROWB>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)));
+        ldmatrix_x4(bf, kt + swz<ROWB>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * (ks + 1) + (lane >> 4)));
+        mma_bf16_16816(sca, af, qb[ks][0], qb[ks][1]);
+        mma_bf16_16816(scb, bf, qb[ks + 1][0], qb[ks + 1][1]);
+    }
+    const int t0 = key0 + g, t1 = t0 + 8;
+    const float x0 = (t0 < L) ? (sca[0] + scb[0]) * scale_log2 : -INFINITY;   // (key t0, head 2tq)
+    const float x1 = (t0 < L) ? (sca[1] + scb[1]) * scale_log2 : -INFINITY;   // (key t0, head 2tq+1)
+    const float x2 = (t1 < L) ? (sca[2] + scb[2]) * scale_log2 : -INFINITY;   // (key t1, head 2tq)
+    const float x3 = (t1 < L) ? (sca[3] + scb[3]) * scale_log2 : -INFINITY;   // (key t1, head 2tq+1)
+    float mx0 = fmaxf(x0, x2), mx1 = fmaxf(x1, x3);
+    if (__any_sync(0xffffffffu, mx0 > m0 + kDecRaise || mx1 > m1 + kDecRaise)) {   // always on a unit's first page
+#pragma unroll
+        for (int d = 4; d <= 16; d <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, d));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, d));
+        }
+        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: key0 < L
+        const float c0 = fast_exp2(m0 - mn0), c1 = fast_exp2(m1 - mn1);
+        m0 = mn0; m1 = mn1;
+        l0 *= c0; l1 *= c1;
+#pragma unroll
+        for (int i = 0; i < KS; ++i) { o[i][0] *= c0; o[i][1] *= c1; o[i][2] *= c0; o[i][3] *= c1; }
+        if (NS > 0) {
+#pragma unroll
+            for (int j = 0; j < (NS > 0 ? NS : 1); ++j) { sm[j][0] *= c0; sm[j][1] *= c1; }
+        }
+    }
+    const float p0 = fast_exp2(x0 - m0), p1 = fast_exp2(x1 - m1);
+    const float p2 = fast_exp2(x2 - m0), p3 = fast_exp2(x3 - m1);
+    l0 += p0 + p2;
+    l1 += p1 + p3;
+
+    if (NS > 0 && probe) {
+#pragma unroll
+        for (int j = 0; j < (NS > 0 ? NS : 1); ++j) {
+            const int sa = span[2 * j], sb = span[2 * j + 1];
+            if (sb > key0 && sa < key0 + kPage) {
+                const bool in0 = (t0 >= sa) && (t0 < sb), in1 = (t1 >= sa) && (t1 < sb);
+                sm[j][0] += (in0 ? p0 : 0.f) + (in1 ? p2 : 0.f);
+                sm[j][1] += (in0 ? p1 : 0.f) + (in1 ? p3 : 0.f);
+            }
+        }
+    }
+
+    // P^T as the B operand (k = key, n = head): transpose the two 8x8 blocks across lanes.
+    const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
+    const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
+#pragma unroll
+    for (int i = 0; i < KS; ++i) {
+        uint32_t af[4];
+        ldmatrix_x4_trans(af, vt + swz<ROWB>((lane & 7) + (lane >> 4) * 8, 2 * i + ((lane >> 3) & 1)));
+        mma_bf16_16816(o[i], af, pb0, pb1);
+    }
+}
+
 template <int HD, int NS>
 __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const KernelArgs a, const HeadCfg hc)
 {
@@ -226,58 +302,7 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_stream_kernel(const Ker
             const uint32_t kt = wbase + (it % kDecStages) * (2 * TILEB);
             const uint32_t vt = kt + TILEB;
 
-            float sc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                uint32_t af[4];
-                ldmatrix_x4(af, kt + swz<ROWB>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)));
-                mma_bf16_16816(sc, af, qb[ks][0], qb[ks][1]);
-            }
-            const int t0 = key0 + g, t1 = t0 + 8;
-            const float x0 = (t0 < L) ? sc[0] * a.scale_log2 : -INFINITY;   // (key t0, head 2tq)
-            const float x1 = (t0 < L) ? sc[1] * a.scale_log2 : -INFINITY;   // (key t0, head 2tq+1)
-            const float x2 = (t1 < L) ? sc[2] * a.scale_log2 : -INFINITY;   // (key t1, head 2tq)
-            const float x3 = (t1 < L) ? sc[3] * a.scale_log2 : -INFINITY;   // (key t1, head 2tq+1)
-            float mx0 = fmaxf(x0, x2), mx1 = fmaxf(x1, x3);
-#pragma unroll
-            for (int d = 4; d <= 16; d <<= 1) {
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, d));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, d));
-            }
-            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: key0 < L
-            const float c0 = fast_exp2(m0 - mn0), c1 = fast_exp2(m1 - mn1);
-            m0 = mn0; m1 = mn1;
-            const float p0 = fast_exp2(x0 - mn0), p1 = fast_exp2(x1 - mn1);
-            const float p2 = fast_exp2(x2 - mn0), p3 = fast_exp2(x3 - mn1);
-            l0 = l0 * c0 + (p0 + p2);
-            l1 = l1 * c1 + (p1 + p3);
-#pragma unroll
-            for (int i = 0; i < KS; ++i) { o[i][0] *= c0; o[i][1] *= c1; o[i][2] *= c0; o[i][3] *= c1; }
-
-            if (NS > 0 && probe) {
-#pragma unroll
-                for (int j = 0; j < NS; ++j) {
-                    const int sa = sh_span[warp][2 * j], sb = sh_span[warp][2 * j + 1];
-                    float add0 = 0.f, add1 = 0.f;
-                    if (sb > key0 && sa < key0 + kPage) {
-                        const bool in0 = (t0 >= sa) && (t0 < sb), in1 = (t1 >= sa) && (t1 < sb);
-                        add0 = (in0 ? p0 : 0.f) + (in1 ? p2 : 0.f);
-                        add1 = (in0 ? p1 : 0.f) + (in1 ? p3 : 0.f);
-                    }
-                    sm[j][0] = sm[j][0] * c0 + add0;
-                    sm[j][1] = sm[j][1] * c1 + add1;
-                }
-            }
-
-            // P^T as the B operand (k = key, n = head): transpose the two 8x8 blocks across lanes.
-            const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
-            const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
-#pragma unroll
-            for (int i = 0; i < KS; ++i) {
-                uint32_t af[4];
-                ldmatrix_x4_trans(af, vt + swz<ROWB>((lane & 7) + (lane >> 4) * 8, 2 * i + ((lane >> 3) & 1)));
-                mma_bf16_16816(o[i], af, pb0, pb1);
-            }
+            decode_page<HD, NS>(kt, vt, key0, L, a.scale_log2, probe, sh_span[warp], qb, m0, m1, l0, l1, o, sm);
             __syncwarp();
         }
         cp_async_wait<0>();
@@ -430,58 +455,7 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_splitk_kernel(const Ker
         const uint32_t kt = wbase + (it % kDecStages) * (2 * TILEB);
         const uint32_t vt = kt + TILEB;
 
-        float sc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            uint32_t af[4];
-            ldmatrix_x4(af, kt + swz<ROWB>((lane & 7) + ((lane >> 3) & 1) * 8, 2 * ks + (lane >> 4)));
-            mma_bf16_16816(sc, af, qb[ks][0], qb[ks][1]);
-        }
-        const int t0 = key0 + g, t1 = t0 + 8;
-        const float x0 = (t0 < L) ? sc[0] * a.scale_log2 : -INFINITY;   // (key t0, head 2tq)
-        const float x1 = (t0 < L) ? sc[1] * a.scale_log2 : -INFINITY;   // (key t0, head 2tq+1)
-        const float x2 = (t1 < L) ? sc[2] * a.scale_log2 : -INFINITY;   // (key t1, head 2tq)
-        const float x3 = (t1 < L) ? sc[3] * a.scale_log2 : -INFINITY;   // (key t1, head 2tq+1)
-        float mx0 = fmaxf(x0, x2), mx1 = fmaxf(x1, x3);
-#pragma unroll
-        for (int d = 4; d <= 16; d <<= 1) {
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, d));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, d));
-        }
-        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: key0 < L
-        const float c0 = fast_exp2(m0 - mn0), c1 = fast_exp2(m1 - mn1);
-        m0 = mn0; m1 = mn1;
-        const float p0 = fast_exp2(x0 - mn0), p1 = fast_exp2(x1 - mn1);
-        const float p2 = fast_exp2(x2 - mn0), p3 = fast_exp2(x3 - mn1);
-        l0 = l0 * c0 + (p0 + p2);
-        l1 = l1 * c1 + (p1 + p3);
-#pragma unroll
-        for (int i = 0; i < KS; ++i) { o[i][0] *= c0; o[i][1] *= c1; o[i][2] *= c0; o[i][3] *= c1; }
-
-        if (NS > 0 && probe) {
-#pragma unroll
-            for (int j = 0; j < NS; ++j) {
-                const int sa = sh_span[2 * j], sb = sh_span[2 * j + 1];
-                float add0 = 0.f, add1 = 0.f;
-                if (sb > key0 && sa < key0 + kPage) {
-                    const bool in0 = (t0 >= sa) && (t0 < sb), in1 = (t1 >= sa) && (t1 < sb);
-                    add0 = (in0 ? p0 : 0.f) + (in1 ? p2 : 0.f);
-                    add1 = (in0 ? p1 : 0.f) + (in1 ? p3 : 0.f);
-                }
-                sm[j][0] = sm[j][0] * c0 + add0;
-                sm[j][1] = sm[j][1] * c1 + add1;
-            }
-        }
-
-        // P^T as the B operand (k = key, n = head): transpose the two 8x8 blocks across lanes.
-        const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
-        const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
-#pragma unroll
-        for (int i = 0; i < KS; ++i) {
-            uint32_t af[4];
-            ldmatrix_x4_trans(af, vt + swz<ROWB>((lane & 7) + (lane >> 4) * 8, 2 * i + ((lane >> 3) & 1)));
-            mma_bf16_16816(o[i], af, pb0, pb1);
-        }
+        decode_page<HD, NS>(kt, vt, key0, L, a.scale_log2, probe, sh_span, qb, m0, m1, l0, l1, o, sm);
         __syncwarp();
     }
     cp_async_wait<0>();
