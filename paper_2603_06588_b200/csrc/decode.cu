@@ -9,7 +9,7 @@
 //   units the hardware's CTA dispatch keeps every SM busy and evens out their speeds.
 // * decode_stream (few units, long sequences): fixed chunks would mean either too few CTAs or many
 //   short ones and a large merge.  Here the 16-key pages of all units form one flat list
-//   (sequence-major, then KV head, then page) and every warp of a grid of two CTAs per SM takes an
+//   (sequence-major, then KV head, then page) and every warp of a grid of three CTAs per SM takes an
 //   equal, contiguous share of it, found from the sequence lengths on the device.  A warp walks its
 //   share unit by unit and writes one partial per unit it touches to slot `unit + warp` (both grow
 //   along the walk, so the slot is unique).
@@ -28,12 +28,18 @@
 namespace hook_attn {
 
 constexpr int kDecWarps = 4;
-constexpr int kDecStages = 3;
-constexpr int kDecCtas = 2 * 148;                     // grid of the streaming kernel: two CTAs on each SM of a B200
+// Two stages of one page (K and V) per warp: 64 KB per CTA, three CTAs per SM.  A warp needs well over
+// a thousand cycles per page (dependent MMA chains, the exponentials, the transposes), so twelve warps
+// per SM with one page in flight each stream faster than eight with two (measured: decode batch 104.4
+// against 108.4 us per step; four warps with five pages in flight each: 145.6 us).
+constexpr int kDecStages = 2;
+constexpr int kDecCtasPerSM = 3;
+constexpr int kDecCtas = kDecCtasPerSM * 148;         // grid of the streaming kernel: as many CTAs as a B200 holds
+constexpr int kDecStreamUnits = 2 * 148;              // the streaming kernel is picked for fewer units than this
 constexpr int kDecWorkers = kDecCtas * kDecWarps;     // its warps, which share the flat page list
 constexpr int kScanSeqs = 512;                        // most sequences the streaming kernel is picked for (a power of two)
 constexpr int kPartPad = 16;   // floats after o[D] in a partial: m, l, s[0..7], padding
-static_assert(kDecCtas <= kScanSeqs, "the streaming kernel is picked for fewer than kDecCtas units");
+static_assert(kDecStreamUnits <= kScanSeqs, "the streaming kernel scans all sequences in one pass");
 
 template <int HD>
 constexpr int decode_smem_bytes()
@@ -639,7 +645,7 @@ struct DecodePlan {
 static DecodePlan decode_plan(int num_seqs, int Hkv, int max_blocks)
 {
     DecodePlan p = {};
-    p.stream = (long)num_seqs * Hkv < kDecCtas;
+    p.stream = (long)num_seqs * Hkv < kDecStreamUnits;
     const long max_keys = (long)max_blocks * kPage;
     p.chunk = 2048;
     while (p.chunk > 256) {
