@@ -55,8 +55,8 @@ WORKLOADS = {
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu captures
 # summarised under profiles/ (None where no capture of the current kernel exists).
 DRAM_TRAFFIC = {
-    "cfg2_decode": 625.11e6 + 6.70e6,     # profiles/decode_splitk_kernel__cfg2_decode.md
-    "cfg5_decode": 538.10e6 + 4.26e6,     # profiles/decode_stream_kernel__cfg5_decode.md
+    "cfg2_decode": 625.09e6 + 6.98e6,     # profiles/decode_splitk_kernel__cfg2_decode.md
+    "cfg5_decode": 538.10e6 + 5.82e6,     # profiles/decode_stream_kernel__cfg5_decode.md
     "cfg3_prefill_small": 50.42e6 + 4.53e6,   # profiles/prefill_tc_kernel__cfg3_prefill_small.md
 }
 
