@@ -81,17 +81,18 @@ cudaError_t launch_steer_residual(__nv_bfloat16* hidden, const float* vec, float
 }
 
 // ---- raw q/k capture ----------------------------------------------------------------------------
-// k: grid (key tiles of 64, sequences); every 16 lanes move one (key, probed head) row of D bf16
-// with 16-byte accesses through the block table.  q: one (row, probed head) per 16 lanes.
+// k: grid (key tiles of 64, sequences); a warp takes one key at a time.  The key's rows of all KV heads
+// are contiguous in the cache and its rows of the P probed heads are contiguous in the output, so the warp
+// looks the page up once and then moves 32 / (D / 8) rows per instruction with 16-byte accesses (several
+// in flight): no per-row index arithmetic.  q: one (row, probed head) per 16 lanes.
 template <int HD>
 __global__ void __launch_bounds__(256) capture_k_kernel(const KernelArgs a, const HeadCfg hc, __nv_bfloat16* __restrict__ k_out,
                                                         const int32_t* __restrict__ cu_k)
 {
     constexpr int LPR = HD / 8;                 // lanes per row (16-byte packets)
-    __shared__ int8_t sh_heads[kMaxHeads];
-    if (threadIdx.x < kMaxHeads) sh_heads[threadIdx.x] = 0;
-    __syncthreads();
-    if ((int)threadIdx.x < a.Hq && hc.slot[threadIdx.x] >= 0) sh_heads[hc.slot[threadIdx.x]] = (int8_t)threadIdx.x;
+    constexpr int RPW = 32 / LPR;               // rows per warp instruction
+    __shared__ int8_t sh_kvh[kMaxHeads];        // KV head of the probed head in slot i
+    if ((int)threadIdx.x < a.Hq && hc.slot[threadIdx.x] >= 0) sh_kvh[hc.slot[threadIdx.x]] = (int8_t)(threadIdx.x / a.G);
     __syncthreads();
     const int s = blockIdx.y;
     const int L = a.seq_lens[s];
@@ -101,34 +102,29 @@ __global__ void __launch_bounds__(256) capture_k_kernel(const KernelArgs a, cons
     }
     const int t0 = blockIdx.x * 64;
     if (t0 >= L) return;
-    const int nkeys = min(64, L - t0);
-    const int sub = threadIdx.x / LPR, part = threadIdx.x % LPR;
-    const int rows_per_step = 256 / LPR;
+    const int t1 = min(L, t0 + 64);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane / LPR, part = lane % LPR;
     const int32_t* bt = a.block_table + (int64_t)s * a.max_blocks;
-    const int64_t out0 = (int64_t)cu_k[s] + t0;
-    // four rows per thread and step: the loads are issued together, then the stores
-    const int total = nkeys * a.P;
-    for (int r0 = sub; r0 < total; r0 += 4 * rows_per_step) {
-        uint4 v[4];
-        int64_t dst[4];
+    const int64_t out0 = (int64_t)cu_k[s];
+    for (int t = t0 + warp; t < t1; t += 8) {
+        const int page = bt[t / kPage];
+        if (page < 0 || page >= a.num_blocks) { if (lane == 0) report(a.status, HOOK_ATTN_ERR_BOUNDS); continue; }
+        const __nv_bfloat16* src = a.k + (int64_t)page * a.bs + (int64_t)(t % kPage) * a.ts + part * 8;
+        __nv_bfloat16* dst = k_out + (out0 + t) * a.P * HD + part * 8;
+        for (int p0 = 0; p0 < a.P; p0 += 4 * RPW) {   // four instructions' worth of rows: loads first, then stores
+            uint4 v[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int r = r0 + u * rows_per_step;
-            dst[u] = -1;
-            if (r < total) {
-                const int tk = r / a.P, pi = r % a.P;
-                const int t = t0 + tk;
-                const int page = bt[t / kPage];
-                if (page < 0 || page >= a.num_blocks) { report(a.status, HOOK_ATTN_ERR_BOUNDS); continue; }
-                const int kvh = sh_heads[pi] / a.G;
-                v[u] = *reinterpret_cast<const uint4*>(a.k + (int64_t)page * a.bs + (int64_t)(t % kPage) * a.ts +
-                                                       (int64_t)kvh * a.hs + part * 8);
-                dst[u] = ((out0 + tk) * a.P + pi) * HD + part * 8;
+            for (int u = 0; u < 4; ++u) {
+                const int pi = p0 + u * RPW + sub;
+                if (pi < a.P) v[u] = *reinterpret_cast<const uint4*>(src + (int64_t)sh_kvh[pi] * a.hs);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int pi = p0 + u * RPW + sub;
+                if (pi < a.P) *reinterpret_cast<uint4*>(dst + (int64_t)pi * HD) = v[u];
             }
         }
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (dst[u] >= 0) *reinterpret_cast<uint4*>(k_out + dst[u]) = v[u];
     }
 }
 
