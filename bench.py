@@ -1,24 +1,35 @@
 """Benchmark of the hooked paged-attention path.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
 
 A step is one pass of the whole hot path (page resolve, scores, online softmax, span masses, PV,
-steering add, store and -- for decode -- the split-K merge) over one batch of seeded synthetic
-input.  The default workload is the decode batch (64 sequences, contexts 512..4096, 32/8 heads,
-head_dim 128, 16 probed heads, 2 spans, 4 steered heads); `--workload` selects the others.
+steering add, store and -- for decode -- the split-K merge) over one batch of seeded synthetic input.
 
-The printed JSON line carries the whole-job throughput with inputs resident in HBM (`value`), the
-same metric through the public call with host buffers (`e2e`), the roofline of the dominant kernel,
-the hook overhead against the same kernels with hooks disabled, and the fp64 CPU oracle timed on
-the host cores (`cpu_baseline`; a reported baseline, not the target).
+Without ``--workload`` the headline is the long-context workload: one step = one full causal prefill
+call of 4 x 32768 tokens plus the 128 decode steps that follow it on the same cache (64/8 heads,
+head_dim 128, all 64 heads probed on 8 spans, 8 steered heads); ``value`` is tokens (query rows) per
+second over the whole step.  The line also carries a ``workloads`` object with every other named
+workload (decode batch, 32-layer prefill, the mixed batch's decode call, prefill call and both
+together, the long-context prefill and decode step alone, and the long-context session with 16 of
+64 heads probed): per workload the time per step (median of at least five blocks that together run
+for at least half a second, with the spread), the roofline of its dominant kernel, the hook
+overhead against the same kernels with hooks disabled, and the clocks seen while it ran.
 
-With N > 1 (torchrun) every rank runs an independent replica of the workload -- the path has no
-exchange step, so there is no collective on the data path; timing is the max over ranks.
+``e2e`` is the same metric through the public call with HOST buffers: the step's inputs (queries,
+tables, lengths, spans) come from pinned host memory and the results go back to the host every step;
+the KV cache is state that stays resident on the device, as it does while serving.  ``cpu_baseline``
+(and ``--impl reference``) time the fp64 CPU oracle on the host cores on a bounded sample of the
+headline workload: a reported baseline, not the target.
+
+With N > 1 (torchrun) every rank runs an independent replica of the headline workload -- the path has
+no exchange step, so there is no collective on the data path; timing is the max over ranks.
 """
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -37,58 +48,32 @@ from paper_2603_06588_b200 import inputs  # noqa: E402
 METRIC = "hooked-attn tokens/s"
 UNIT = "tokens/s"
 
+HEADLINE = "cfg5_long_context"
 WORKLOADS = {
+    "cfg5_long_context": "long context: 4 seqs x 32768 tokens, one full causal prefill call plus the 128 decode steps that follow "
+                         "on the same cache, Hq64/Hkv8, D128, 64 probed heads, 8 spans, 8 steered heads (alpha 0.8)",
+    "cfg5_16of64": "long context as above with 16 of the 64 heads probed",
+    "cfg5_prefill": "long context, the prefill call alone: 4 seqs x 32768 tokens causal, 64 probed heads, 8 spans, 8 steered heads",
+    "cfg5_decode": "long context, one decode step alone (step 64): 4 seqs at 32833 keys, 64 probed heads, 8 spans, 8 steered heads",
     "cfg2_decode": "decode batch: 64 seqs x 1 token, ctx U[512,4096], Hq32/Hkv8, D128, 16 probed heads, 2 spans, 4 steered heads",
-    "cfg3_prefill": "prefill: 8 seqs x 4096 tokens causal, Hq32/Hkv8, D128, ~10% (layer,head) pairs probed, 3 spans, one layer call per step",
-    "cfg3_prefill_32layers": "prefill: 32 independent layers' worth of seeded inputs (8 seqs x 4096 each), the seeded 10% of the 1024 (layer, head) pairs probed, 3 spans; one step = 32 layer calls",
+    "cfg3_prefill_32layers": "prefill: 32 independent layers' worth of seeded inputs (8 seqs x 4096 tokens each, Hq32/Hkv8, D128), the "
+                             "seeded 10% of the 1024 (layer, head) pairs probed, 3 spans; one step = 32 layer calls",
+    "cfg4_decode": "mixed batch, decode call: 256 seqs, ctx U[1024,8192], Hq28/Hkv4, D128, 14 probed heads, 4 spans, 8 steered heads",
+    "cfg4_prefill": "mixed batch, prefill call: 2 chunks of 2048 tokens on 4096-token contexts, Hq28/Hkv4, D128",
+    "cfg4_mixed": "mixed chunked batch: the 256-sequence decode call and the 2-chunk prefill call of one step together",
+    # profiling sizes and the companions of the attention path (only with --workload)
+    "cfg3_prefill": "prefill: 8 seqs x 4096 tokens causal, Hq32/Hkv8, D128, layer-0 probes, 3 spans, one layer call per step",
     "cfg3_prefill_small": "prefill, profiling size: 2 seqs x 2048 tokens causal, Hq32/Hkv8, D128, layer-0 probes, 3 spans",
-    "cfg4_decode": "mixed batch, decode part: 256 seqs, ctx U[1024,8192], Hq28/Hkv4, D128, 14 probed heads, 4 spans, 8 steered heads",
-    "cfg4_prefill": "mixed batch, prefill part: 2 chunks of 2048 tokens on 4096-token contexts, Hq28/Hkv4, D128",
-    "cfg4_mixed": "mixed chunked batch: the 256-sequence decode call and the 2-chunk prefill call of one step, issued on two streams",
+    "cfg5_decode_small": "long-context decode, profiling size: 4 seqs at 8192 keys, Hq64/Hkv8, D128, 64 probed heads, 8 spans",
     "steer_residual": "residual-stream steering: hidden[32768 x 4096] bf16 += alpha * vec, in place",
     "capture_qk": "raw q/k capture of the 16 probed heads of the decode batch (64 seqs, ctx U[512,4096])",
-    "cfg5_decode": "long context decode: 4 seqs at 32768+ keys, Hq64/Hkv8, D128, 64 probed heads, 8 spans, 8 steered heads",
-    "cfg5_prefill": "long context prefill: 4 seqs x 32768 tokens causal, Hq64/Hkv8, D128, 64 probed heads, 8 spans, 8 steered heads",
 }
-
+TABLE = ["cfg2_decode", "cfg3_prefill_32layers", "cfg4_decode", "cfg4_prefill", "cfg4_mixed", "cfg5_prefill", "cfg5_decode",
+         "cfg5_16of64"]
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu captures
-# summarised under profiles/ (None where no capture of the current kernel exists).
-DRAM_TRAFFIC = {
-    "cfg2_decode": 625.09e6 + 6.98e6,     # profiles/decode_splitk_kernel__cfg2_decode.md
-    "cfg5_decode": 538.10e6 + 5.82e6,     # profiles/decode_stream_kernel__cfg5_decode.md
-    "cfg3_prefill_small": 50.42e6 + 4.53e6,   # profiles/prefill_tc_kernel__cfg3_prefill_small.md
-}
-
-
-def make_workload(name: str):
-    if name == "cfg2_decode":
-        return inputs.config2_decode()
-    if name == "cfg3_prefill":
-        return inputs.config3_prefill(layer=0, force_probe=True)
-    if name == "cfg3_prefill_small":
-        return inputs.config3_prefill(layer=0, num_seqs=2, tokens=2048, force_probe=True)
-    if name == "cfg4_decode":
-        return inputs.config4_decode()
-    if name == "cfg4_prefill":
-        return inputs.config4_prefill()
-    if name == "cfg5_decode":
-        return inputs.config5_decode(step=64)
-    if name == "cfg5_prefill":
-        return inputs.config5_prefill()
-    raise SystemExit(f"unknown workload {name}; choose from {sorted(WORKLOADS)}")
-
-
-def algorithmic_work(case):
-    """Algorithmic bytes and flops of one step: every needed K and V element once per KV head,
-    plus q, out, span_mass and the tables; flops = 4*D per visible (row, key, query head)."""
-    D, Hq, Hkv = case.head_dim, case.num_q_heads, case.num_kv_heads
-    kv_bytes = case.kv_tokens() * Hkv * D * 2 * 2
-    qo_bytes = 2 * case.total_q * Hq * D * 2
-    rows = case.num_seqs if (case.is_decode or case.probe_rows == inputs.PROBE_ROWS_LAST) else case.total_q
-    misc = rows * case.num_probed * case.num_spans * 4 + case.kv_tokens() // inputs.PAGE * 4 + case.num_seqs * 8
-    flops = 4.0 * D * case.visible_pairs() * Hq
-    return kv_bytes + qo_bytes + misc, flops
+# summarised under profiles/ (absent = no capture of the current kernel exists: reported as null).
+DRAM_TRAFFIC = {}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -103,15 +88,25 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def host_cores():
+    """Cores the process may use, the machine's count, and the process's affinity list length."""
+    try:
+        aff = len(os.sched_getaffinity(0))
+    except AttributeError:
+        aff = None
+    return {"sched_getaffinity": aff, "hardware_concurrency": os.cpu_count()}
+
+
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """One `nvidia-smi` process sampling clocks, power and throttle reasons every 100 ms with time stamps;
+    `window(t0, t1)` summarises the samples taken between two wall-clock instants."""
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+    NAMES = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
 
     def __init__(self, index: int):
-        self.index = index
-        self.proc = None
-        self.file = None
+        self.index, self.proc, self.file, self.rows = index, None, None, None
 
     def start(self):
         try:
@@ -123,9 +118,9 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "sm_mhz_min": None, "power_w": None}
+        self.rows = []
         if self.proc is None:
-            return out
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -133,86 +128,350 @@ class ClockSampler:
             self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, mx, pw, reasons = [], [], [], set()
         for line in self.file.read().splitlines():
             f = [x.strip() for x in line.split(",")]
-            if len(f) < 9:
+            if len(f) < 8:
                 continue
             try:
-                sm.append(float(f[1]))
-                mx.append(float(f[2]))
-                pw.append(float(f[3]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                self.rows.append((ts, float(f[1]), float(f[2]), float(f[3]),
+                                  [n for n, v in zip(self.NAMES, f[4:8]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
         self.file.close()
         os.unlink(self.file.name)
-        if sm:
-            # samples under load: the upper half of the observed clocks (idle samples sit low)
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm),
-                       sm_mhz_min=min(sm), power_w=statistics.median(pw) if pw else None)
+
+    def window(self, t0: float, t1: float):
+        rows = [r for r in (self.rows or []) if t0 - 0.05 <= r[0] <= t1 + 0.05]
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": len(rows), "sm_mhz_min": None, "power_w": None}
+        if rows:
+            out.update(sm_mhz=statistics.median(r[1] for r in rows), sm_max_mhz=max(r[2] for r in rows),
+                       sm_mhz_min=min(r[1] for r in rows), power_w=statistics.median(r[3] for r in rows),
+                       reasons=sorted({n for r in rows for n in r[4]}))
         return out
 
 
 # ------------------------------------------------------------------------------------------------
-def run_reference(args):
-    """The oracle, as it stands, timed on the host cores on the same workload and metric."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
-    from oracle import oracle
-    case = make_workload(args.workload)
-    # every step is a bounded sample, sized so that the whole run ends within a few minutes
-    budget = min(args.ref_budget, 120.0 / max(1, args.steps + args.warmup))
-    rows, desc, scale_tokens = oracle_sample(case, budget_s=budget)
-    for _ in range(args.warmup):
-        oracle.run(case, rows=rows)
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        oracle.run(case, rows=rows)
-    dt = (time.perf_counter() - t0) / args.steps
-    tokens = scale_tokens
-    val = tokens / dt
-    line = {
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}"},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": desc},
-        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-    }
-    print(json.dumps(line))
+# timing
+def _event_pair():
+    return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
 
-def oracle_sample(case, budget_s: float):
-    """A bounded sample of the workload for the CPU oracle: global query rows, a description, and
-    the number of tokens the timing is scaled to (rows evaluated, weighted by visible keys so that
-    the figure stays a tokens/s of the same workload)."""
-    total_pairs = case.visible_pairs()
-    # the oracle sustains very roughly 5e8 (key, d) multiply-adds per core-second over K and V
-    macs_per_row_key = 2 * case.head_dim * case.num_q_heads
-    budget_pairs = budget_s * 5e8 * max(1, os.cpu_count() or 1) / macs_per_row_key
-    if total_pairs <= budget_pairs:
-        return list(range(case.total_q)), f"all {case.total_q} query rows x {case.num_q_heads} heads", case.total_q
-    rows = inputs.sample_rows(case, extra_random=256)
-    cu = case.cu_q_lens.tolist()
-    Ls = case.seq_lens.tolist()
+def time_blocks(step_fns, warmup: int, blocks: int = 5, min_total: float = 0.5, steps_per_block: int = 0, sync=None):
+    """Time one or several step functions in interleaved blocks (fn0 block, fn1 block, fn0 block, ...), CUDA
+    events on the current stream, a synchronize on both sides of every block.  Returns per function the list
+    of seconds per step of its blocks, plus the steps per block and the wall-clock window of the whole."""
+    sync = sync or torch.cuda.synchronize
+    for fn in step_fns:
+        for _ in range(max(1, warmup)):
+            fn()
+    e0, e1 = _event_pair()
+    sync()
+    if steps_per_block <= 0:
+        e0.record()
+        step_fns[0]()
+        e1.record()
+        e1.synchronize()
+        t1 = max(e0.elapsed_time(e1) / 1e3, 1e-6)
+        steps_per_block = max(1, math.ceil(min_total / blocks / t1))
+    times = [[] for _ in step_fns]
+    w0 = time.time()
+    for _ in range(blocks):
+        for i, fn in enumerate(step_fns):
+            sync()
+            e0.record()
+            for _ in range(steps_per_block):
+                fn()
+            e1.record()
+            e1.synchronize()
+            times[i].append(e0.elapsed_time(e1) / 1e3 / steps_per_block)
+    sync()
+    return times, steps_per_block, (w0, time.time())
+
+
+def stats(ts):
+    return {"ms_per_step": statistics.median(ts) * 1e3, "ms_min": min(ts) * 1e3, "ms_max": max(ts) * 1e3, "blocks": len(ts)}
+
+
+def algorithmic_work(case):
+    """Algorithmic bytes and flops of one call: every needed K and V element once per KV head, plus q,
+    out, span_mass and the tables; flops = 4*D per visible (row, key, query head)."""
+    D, Hq, Hkv = case.head_dim, case.num_q_heads, case.num_kv_heads
+    kv_bytes = case.kv_tokens() * Hkv * D * 2 * 2
+    qo_bytes = 2 * case.total_q * Hq * D * 2
+    rows = case.num_seqs if (case.is_decode or case.probe_rows == inputs.PROBE_ROWS_LAST) else case.total_q
+    misc = rows * case.num_probed * case.num_spans * 4 + case.kv_tokens() // inputs.PAGE * 4 + case.num_seqs * 8
+    flops = 4.0 * D * case.visible_pairs() * Hq
+    return kv_bytes + qo_bytes + misc, flops
+
+
+def roofline(bound, work, seconds, peaks, kernel, region_s, traffic=None):
+    """`work` = algorithmic bytes (hbm) or flops (tensor) of the launches that took `seconds`."""
+    if bound == "hbm":
+        achieved, peak, unit, kind = work / seconds / 1e9, peaks["hbm_gbs"], "GB/s", "copy bandwidth"
+        extra = {"algorithmic_bytes": work, "frac_of_datasheet": achieved / 8000.0}
+    else:
+        achieved, unit = work / seconds / 1e12, "TFLOP/s"
+        sustained = region_s >= 2.0          # seconds of back-to-back tensor work: the board sits at its power cap
+        peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+        kind = "bf16 GEMM, sustained (timed region of %.1f s)" % region_s if sustained else "bf16 GEMM, burst (timed region of %.1f s)" % region_s
+        extra = {"algorithmic_flops": work, "frac_of_burst": achieved / peaks["bf16_tflops"],
+                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"], "frac_of_datasheet": achieved / 2250.0}
+    out = {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak, "traffic": traffic,
+           "peak_source": f"of {peaks['source']} ({kind})", "kernel": kernel}
+    out.update(extra)
+    return out
+
+
+def decode_kernel_name(case):
+    first = "decode_stream_kernel" if case.num_seqs * case.num_kv_heads < 296 else "decode_splitk_kernel"
+    return first + " (+ decode_merge_kernel; duration = the whole call, conservative)"
+
+
+# ------------------------------------------------------------------------------------------------
+# workloads: each builder returns a dict with the hooked and the plain step and what one step does
+class Ctx:
+    def __init__(self, eng, device, peaks):
+        self.eng, self.device, self.peaks = eng, device, peaks
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def plans(self, case, binding):
+        """(hooked plan, plain plan) of a case: same device tensors, hooks disabled in the second."""
+        kw = binding.case_to_device(case, self.device)
+        hooked = self.eng.plan(case.is_decode, status=self.status, **kw)
+        off = case.without_hooks()
+        kw_off = {k: v for k, v in kw.items() if k not in ("spans", "head_mask", "alpha", "steer_vec")}
+        plain = self.eng.plan(off.is_decode, status=self.status, out=hooked.out, **kw_off)
+        return hooked, plain
+
+
+def build_single(ctx, case, binding):
+    hooked, plain = ctx.plans(case, binding)
+    b, f = algorithmic_work(case)
+    bound = "hbm" if case.is_decode else "tensor"
+    return {"hooked": hooked.run, "plain": plain.run, "tokens": case.total_q, "bound": bound,
+            "work": b if bound == "hbm" else f, "kernel": decode_kernel_name(case) if case.is_decode else "prefill_tc_kernel",
+            "launches": 2 if case.is_decode else 1, "keep": (hooked, plain), "case": case}
+
+
+def build_layers(ctx, binding, layers=32):
+    hooked, plain, flops, probed, tokens = [], [], 0.0, 0, 0
+    for layer in range(layers):
+        case = inputs.config3_prefill(layer=layer, device=ctx.device)
+        if case.num_probed == 0:
+            case = case.without_hooks()
+        probed += case.num_probed
+        h, p = ctx.plans(case, binding)
+        hooked.append(h)
+        plain.append(p)
+        flops += algorithmic_work(case)[1]
+        tokens += case.total_q
+
+    def run(plans):
+        def step():
+            for p in plans:
+                p.run()
+        return step
+    return {"hooked": run(hooked), "plain": run(plain), "tokens": tokens, "bound": "tensor", "work": flops,
+            "kernel": "prefill_tc_kernel (32 launches per step)", "launches": layers, "keep": (hooked, plain),
+            "extra": {"layers": layers, "probed_layer_head_pairs": probed}}
+
+
+def build_mixed(ctx, binding):
+    dec, pf = inputs.config4_decode(device=ctx.device), inputs.config4_prefill(device=ctx.device)
+    dh, dp = ctx.plans(dec, binding)
+    ph, pp = ctx.plans(pf, binding)
+    side = torch.cuda.Stream(device=ctx.device)
+    fork, join = torch.cuda.Event(), torch.cuda.Event()
+
+    def both(d, p):
+        def step():
+            main_s = torch.cuda.current_stream()
+            fork.record(main_s)
+            side.wait_event(fork)
+            with torch.cuda.stream(side):
+                p.run()
+                join.record(side)
+            d.run()
+            main_s.wait_event(join)
+        return step
+    bytes_dec, _ = algorithmic_work(dec)
+    _, flops_pf = algorithmic_work(pf)
+    return {"hooked": both(dh, ph), "plain": both(dp, pp), "tokens": dec.total_q + pf.total_q, "bound": "hbm", "work": bytes_dec,
+            "kernel": "decode_splitk_kernel + decode_merge_kernel on one stream, prefill_tc_kernel on a second; the bytes are "
+                      "the decode call's, over the time of the whole step",
+            "launches": 3, "keep": (dh, dp, ph, pp), "extra": {"prefill_flops_per_step": flops_pf}}
+
+
+class Session:
+    """The long-context session: one prefill call and the decode steps that follow on the same cache."""
+
+    def __init__(self, ctx, binding, probed=64, steps=128):
+        self.ctx = ctx
+        self.prefill, self.decodes = inputs.config5_session(steps=steps, probed=probed, device=ctx.device)
+        self.pf_h, self.pf_p = ctx.plans(self.prefill, binding)
+        kw = binding.case_to_device(self.decodes[0], ctx.device)
+        self.dec_len = [c.seq_lens.to(ctx.device) for c in self.decodes]
+        first = ctx.eng.plan(True, status=ctx.status, **kw)
+        self.dec_h, self.dec_p = [first], []
+        kw_off = {k: v for k, v in kw.items() if k not in ("spans", "head_mask", "alpha", "steer_vec")}
+        for t, L in enumerate(self.dec_len):
+            if t:
+                self.dec_h.append(ctx.eng.plan(True, status=ctx.status, out=first.out, span_mass=first.span_mass,
+                                               **dict(kw, seq_lens=L)))
+            self.dec_p.append(ctx.eng.plan(True, status=ctx.status, out=first.out, **dict(kw_off, seq_lens=L)))
+        self.tokens = self.prefill.total_q + sum(c.total_q for c in self.decodes)
+        self.flops_pf = algorithmic_work(self.prefill)[1]
+        self.bytes_dec = sum(algorithmic_work(c)[0] for c in self.decodes)
+        self.launches = 1 + 2 * len(self.decodes)
+        self.pf_events = []       # (start, end) events around the prefill call of every hooked step
+
+    def step(self, hooked=True, record=False):
+        pf = self.pf_h if hooked else self.pf_p
+        if record:
+            e0, e1 = _event_pair()
+            e0.record()
+            pf.run()
+            e1.record()
+            self.pf_events.append((e0, e1))
+        else:
+            pf.run()
+        for p in (self.dec_h if hooked else self.dec_p):
+            p.run()
+
+    def prefill_seconds(self):
+        """Average duration of the prefill launches recorded since the last call."""
+        ts = [a.elapsed_time(b) / 1e3 for a, b in self.pf_events]
+        self.pf_events = []
+        return sum(ts) / len(ts)
+
+    def entry(self):
+        return {"hooked": lambda: self.step(True), "plain": lambda: self.step(False), "tokens": self.tokens, "bound": "tensor",
+                "work": None, "kernel": "prefill_tc_kernel (one launch per step, timed by its own events inside the step)",
+                "launches": self.launches, "session": self}
+
+
+def build(ctx, name, binding):
+    dev = ctx.device
+    if name == "cfg2_decode":
+        return build_single(ctx, inputs.config2_decode(device=dev), binding)
+    if name == "cfg3_prefill":
+        return build_single(ctx, inputs.config3_prefill(layer=0, force_probe=True, device=dev), binding)
+    if name == "cfg3_prefill_small":
+        return build_single(ctx, inputs.config3_prefill(layer=0, num_seqs=2, tokens=2048, force_probe=True, device=dev), binding)
+    if name == "cfg3_prefill_32layers":
+        return build_layers(ctx, binding)
+    if name == "cfg4_decode":
+        return build_single(ctx, inputs.config4_decode(device=dev), binding)
+    if name == "cfg4_prefill":
+        return build_single(ctx, inputs.config4_prefill(device=dev), binding)
+    if name == "cfg4_mixed":
+        return build_mixed(ctx, binding)
+    if name == "cfg5_decode_small":
+        return build_single(ctx, inputs.config5_decode(tokens=8192, step=0, device=dev), binding)
+    raise SystemExit(f"unknown workload {name}; choose from {sorted(WORKLOADS)}")
+
+
+def measure_entry(ctx, name, w, warmup, sampler_windows, steps_per_block=0, blocks=5, sync=None):
+    """Times the hooked and the plain step of a workload in interleaved blocks; returns its table entry."""
+    sess = w.get("session")
+    hooked = (lambda: sess.step(True, record=True)) if sess else w["hooked"]
+    region0 = time.time()
+    (th, tp), spb, window = time_blocks([hooked, w["plain"]], warmup=warmup, blocks=blocks, steps_per_block=steps_per_block,
+                                        sync=sync)
+    region_s = (time.time() - region0)
+    sampler_windows[name] = window
+    st = stats(th)
+    per_step = st["ms_per_step"] / 1e3
+    if sess:
+        sess.pf_events = sess.pf_events[-blocks * spb:]     # drop the warm-up launches
+        t_pf = sess.prefill_seconds()
+        roof = roofline("tensor", sess.flops_pf, t_pf, ctx.peaks, w["kernel"], region_s, DRAM_TRAFFIC.get("cfg5_prefill"))
+        roof["launch_ms"] = t_pf * 1e3
+        extra = {"prefill_ms": t_pf * 1e3, "decode_ms_per_step": (per_step - t_pf) * 1e3 / len(sess.decodes),
+                 "decode_gbs": sess.bytes_dec / max(per_step - t_pf, 1e-9) / 1e9}
+    else:
+        roof = roofline(w["bound"], w["work"], per_step, ctx.peaks, w["kernel"], region_s, DRAM_TRAFFIC.get(name))
+        extra = dict(w.get("extra", {}))
+        if "prefill_flops_per_step" in extra:
+            extra["prefill_tflops_over_the_step"] = extra.pop("prefill_flops_per_step") / per_step / 1e12
+    # median of the ratios of neighbouring (hooked, plain) blocks: clock drift moves both members of a pair alike
+    overhead = statistics.median(h / p for h, p in zip(th, tp)) - 1.0
+    entry = {"workload": WORKLOADS[name], "tokens_per_step": w["tokens"], "tokens_per_s": w["tokens"] / per_step}
+    entry.update(st)
+    entry.update({"steps_per_block": spb, "ms_per_step_hooks_off": statistics.median(tp) * 1e3, "hook_overhead": overhead,
+                  "roofline": roof, "gpu_launches_per_step": w["launches"]})
+    entry.update(extra)
+    if int(ctx.status.item()) != 0:
+        raise SystemExit(f"{name}: device status {int(ctx.status.item())}")
+    return entry, th
+
+
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle on a bounded sample of the headline workload
+def oracle_sample(prefill, decode_mid, budget_s: float, cores: int):
+    """Rows of the prefill call (a seeded sample) and one decode step (all its rows), sized for about
+    `budget_s` seconds of oracle time; returns the two row lists and the visible (row, key) pairs per head."""
+    macs_per_pair = 2 * prefill.head_dim * prefill.num_q_heads
+    budget_pairs = budget_s * 5e8 * max(1, cores) / macs_per_pair      # the oracle sustains roughly 5e8 MAC/s per core
+    rows = inputs.sample_rows(prefill, extra_random=64)
+    cu, Ls = prefill.cu_q_lens.tolist(), prefill.seq_lens.tolist()
     order = torch.randperm(len(rows), generator=torch.Generator().manual_seed(11)).tolist()
+    dec_pairs = int(decode_mid.seq_lens.sum())
     picked, pairs = [], 0
     for idx in order:
         r = rows[idx]
-        s = max(i for i in range(case.num_seqs) if cu[i] <= r and cu[i + 1] > cu[i])
+        s = max(i for i in range(prefill.num_seqs) if cu[i] <= r and cu[i + 1] > cu[i])
         pos = Ls[s] - (cu[s + 1] - cu[s]) + (r - cu[s])
-        if pairs + pos + 1 > budget_pairs and picked:
+        if pairs + pos + 1 > budget_pairs - dec_pairs and picked:
             break
         picked.append(r)
         pairs += pos + 1
     picked.sort()
-    tokens = case.total_q * pairs / total_pairs
-    return picked, (f"{len(picked)} sampled query rows x {case.num_q_heads} heads ({pairs} of {total_pairs} visible pairs per head); "
-                    "tokens/s extrapolated by visible-pair count"), tokens
+    return picked, pairs, dec_pairs
+
+
+def run_oracle_sample(sess_cases, budget_s, reps):
+    """Time the oracle on the sample; returns (tokens/s extrapolated by visible pairs, seconds per pass, description)."""
+    from oracle import oracle
+    prefill, decodes = sess_cases
+    cores = oracle.threads()
+    mid = decodes[len(decodes) // 2]
+    rows, pf_pairs, dec_pairs = oracle_sample(prefill, mid, budget_s, cores)
+    total_pairs = prefill.visible_pairs() + sum(int(c.seq_lens.sum()) for c in decodes)
+    tokens = prefill.total_q + sum(c.total_q for c in decodes)
+    host_pf, host_mid = inputs.to_host(prefill), inputs.to_host(mid)
+    oracle.run(host_mid)                                                   # warm-up (threads, page cache)
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle.run(host_pf, rows=rows)
+        oracle.run(host_mid)
+    dt = (time.perf_counter() - t0) / reps
+    frac = (pf_pairs + dec_pairs) / total_pairs
+    desc = (f"{len(rows)} sampled prefill rows + the {mid.total_q} rows of decode step {len(decodes) // 2}, all {prefill.num_q_heads} heads "
+            f"({pf_pairs + dec_pairs} of {total_pairs} visible (row, key) pairs per head); tokens/s extrapolated by visible-pair count")
+    return tokens * frac / dt, dt, desc, cores
+
+
+def run_reference(args):
+    """The oracle, as it stands, timed on the host cores on the headline workload and metric."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    dev = "cuda" if torch.cuda.is_available() else "cpu"       # where the inputs are drawn; the oracle runs on the host
+    cases = inputs.config5_session(device=dev)
+    budget = min(args.ref_budget, 150.0 / max(1, args.steps + args.warmup))
+    for _ in range(args.warmup):
+        run_oracle_sample(cases, budget, 1)
+    val, dt, desc, cores = run_oracle_sample(cases, budget, args.steps)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{HEADLINE}: {WORKLOADS[HEADLINE]}"},
+        "cpu_baseline": dict({"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}, **host_cores()),
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------------------------------
@@ -254,224 +513,97 @@ def run_extra(args):
             torch.cuda.current_stream().synchronize()
         h2d, d2h = 0, k_out.numel() * 2
 
-    def timed(fn, n):
-        for _ in range(args.warmup):
-            fn()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(n):
-            fn()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / 1e3 / n
-
     sampler = ClockSampler(0)
     sampler.start()
-    t = timed(step, args.steps)
-    clocks = sampler.stop()
-    t_e2e = timed(e2e, max(5, min(args.steps, 50)))
+    (ts,), spb, window = time_blocks([step], warmup=args.warmup)
+    (te,), _, _ = time_blocks([e2e], warmup=2, blocks=3, min_total=0.3)
+    sampler.stop()
+    t, t_e2e = statistics.median(ts), statistics.median(te)
     peaks = load_peaks()
-    achieved = alg_bytes / t / 1e9
-    print(json.dumps({
-        "metric": METRIC, "value": tokens / t, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic",
-        "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}", "l2": "inputs larger than L2"},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": f"of {peaks['source']}",
-                     "kernel": kernel, "algorithmic_bytes": alg_bytes},
-        "e2e": {"value": tokens / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": t_e2e * 1e3},
-        "gpu_launches": launches * args.steps,
-        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                   "samples": clocks["samples"]},
-    }))
-
-
-# ------------------------------------------------------------------------------------------------
-def run_layers(args):
-    """The 32-layer prefill workload: every layer has its own seeded q/K/V, block table, spans and head
-    mask (layers without a probed head run with hooks off).  One step = 32 layer calls back to back."""
-    from paper_2603_06588_b200 import binding
-    args.warmup = max(args.warmup, 3)
-    torch.cuda.set_device(0)
-    eng = binding.HookAttn(0)
-    plans, flops, tokens, probed = [], 0.0, 0, 0
-    for layer in range(args.layers):
-        case = inputs.config3_prefill(layer=layer)
-        if case.num_probed == 0:
-            case = case.without_hooks()
-        probed += case.num_probed
-        plans.append(eng.plan(False, **binding.case_to_device(case)))
-        flops += algorithmic_work(case)[1]
-        tokens = case.total_q
-    for p in plans:
-        p.run()
-    torch.cuda.synchronize()
-
-    def step():
-        for p in plans:
-            p.run()
-
-    for _ in range(args.warmup):
-        step()
-    sampler = ClockSampler(0)
-    sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    t = e0.elapsed_time(e1) / 1e3 / args.steps
-    peaks = load_peaks()
-    peak = peaks["bf16_tflops"] if t * args.steps < 2.0 else peaks["bf16_tflops_sustained"]
-    achieved = flops / t / 1e12
-    print(json.dumps({
-        "metric": METRIC, "value": tokens * args.layers / t, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": t * 1e3, "ms_per_layer_call": t * 1e3 / args.layers,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"cfg3_prefill_32layers: {WORKLOADS['cfg3_prefill_32layers']}", "layers": args.layers,
-                   "probed_layer_head_pairs": probed, "l2": "inputs larger than L2 (0.67 GB per layer call)"},
-        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                     "traffic": None, "peak_source": f"of {peaks['source']}", "kernel": "prefill_tc_kernel",
-                     "algorithmic_flops": flops, "frac_of_datasheet": achieved / 2250.0},
-        "e2e": None, "gpu_launches": args.layers * args.steps,
-        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                   "samples": clocks["samples"], "power_w": clocks["power_w"]},
-    }))
-
-
-# ------------------------------------------------------------------------------------------------
-def run_mixed(args):
-    """The mixed chunked batch: one decode call (256 sequences) and one prefill call (2 chunks of 2048
-    rows) per step.  The decode call is HBM-bound and the prefill call tensor-bound, so the step issues
-    them on two streams; the line also reports both calls alone and the gain from the overlap."""
-    from paper_2603_06588_b200 import binding
-    args.warmup = max(args.warmup, 3)
-    torch.cuda.set_device(0)
-    eng = binding.HookAttn(0)
-    dec, pf = inputs.config4_decode(), inputs.config4_prefill()
-    plans, host, devs = {}, {}, {}
-    for name, case in (("dec", dec), ("pf", pf)):
-        kw = binding.case_to_device(case)
-        plans[name] = eng.plan(case.is_decode, **kw)
-        plans[name].run()
-        host[name] = {k: kw[k].cpu().pin_memory() for k in ("q", "block_table", "seq_lens", "cu_q_lens", "spans") if k in kw}
-        devs[name] = kw
-    torch.cuda.synchronize()
-    side = torch.cuda.Stream()
-    fork, join = torch.cuda.Event(), torch.cuda.Event()
-
-    def step_mixed():
-        main_s = torch.cuda.current_stream()
-        fork.record(main_s)
-        side.wait_event(fork)
-        with torch.cuda.stream(side):
-            plans["pf"].run()
-            join.record(side)
-        plans["dec"].run()
-        main_s.wait_event(join)
-
-    def timed(fn, n):
-        for _ in range(args.warmup):
-            fn()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for _ in range(n):
-            fn()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / 1e3 / n
-
-    sampler = ClockSampler(0)
-    sampler.start()
-    t_mixed = timed(step_mixed, args.steps)
-    clocks = sampler.stop()
-    t_dec = timed(plans["dec"].run, args.steps)
-    t_pf = timed(plans["pf"].run, args.steps)
-
-    outs = {n: (torch.empty(plans[n].out.shape, dtype=torch.bfloat16).pin_memory(),
-                torch.empty(plans[n].span_mass.shape, dtype=torch.float32).pin_memory()) for n in plans}
-
-    def step_e2e():
-        for n in plans:
-            for k, t in host[n].items():
-                devs[n][k].copy_(t, non_blocking=True)
-        step_mixed()
-        for n in plans:
-            outs[n][0].copy_(plans[n].out, non_blocking=True)
-            outs[n][1].copy_(plans[n].span_mass, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
-
-    t_e2e = timed(step_e2e, max(10, min(args.steps, 200)))
-    h2d = sum(t.numel() * t.element_size() for n in host for t in host[n].values())
-    d2h = sum(o.numel() * o.element_size() + m.numel() * 4 for o, m in outs.values())
-    peaks = load_peaks()
-    tokens = dec.total_q + pf.total_q
-    bytes_dec, _ = algorithmic_work(dec)
-    _, flops_pf = algorithmic_work(pf)
-    achieved = bytes_dec / t_dec / 1e9
-    line = {
-        "metric": METRIC, "value": tokens / t_mixed, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": t_mixed * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic",
-        "config": {"workload": f"cfg4_mixed: {WORKLOADS['cfg4_mixed']}", "l2": "inputs larger than L2 (2.5 GB per step)",
-                   "kv_cache": "resident in HBM (state, not a per-step input)"},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": f"of {peaks['source']}",
-                     "kernel": "decode_splitk_kernel (+ merge), timed alone: it carries 2.5 GB of the step's bytes",
-                     "algorithmic_bytes": bytes_dec},
-        "mixed": {"decode_alone_ms": t_dec * 1e3, "prefill_alone_ms": t_pf * 1e3, "two_stream_ms": t_mixed * 1e3,
-                  "gain_over_back_to_back": (t_dec + t_pf) / t_mixed,
-                  "prefill_tflops_alone": flops_pf / t_pf / 1e12},
-        "e2e": {"value": tokens / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": t_e2e * 1e3},
-        "gpu_launches": 3 * args.steps,
-        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                   "samples": clocks["samples"]},
-    }
+    line = {"metric": METRIC, "value": tokens / t, "unit": UNIT, "n_gpus": 1, "steps": spb * len(ts), "warmup": args.warmup,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}", "l2": "inputs larger than L2"},
+            "roofline": roofline("hbm", alg_bytes, t, peaks, kernel, 0.0),
+            "e2e": {"value": tokens / t_e2e, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": t_e2e * 1e3},
+            "gpu_launches": launches * spb * len(ts), "clocks": sampler.window(*window)}
+    line.update(stats(ts))
     print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------------------------------
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", default="cfg2_decode")
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--ref-budget", type=float, default=2.0, help="seconds of CPU time per oracle step")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--layers", type=int, default=32, help="layers of the cfg3_prefill_32layers workload")
-    args = ap.parse_args()
-    if args.workload not in WORKLOADS:
-        raise SystemExit(f"unknown workload {args.workload}; choose from {sorted(WORKLOADS)}")
-    if args.impl == "reference":
-        run_reference(args)
-        return
-    from paper_2603_06588_b200.csrc import build as cuda_build
-    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
-        cuda_build.build()      # no-op when the in-tree library is up to date
-    if args.workload == "cfg3_prefill_32layers":
-        run_layers(args)
-        return
-    if args.workload in ("steer_residual", "capture_qk"):
-        run_extra(args)
-        return
-    if args.workload == "cfg4_mixed":
-        if int(os.environ.get("WORLD_SIZE", "1")) > 1:
-            raise SystemExit("cfg4_mixed is a single-GPU measurement")
-        run_mixed(args)
-        return
-    args.warmup = max(args.warmup, 3)
-
+def run_one(args):
+    """A single named workload (profiling sizes, or one row of the table by itself)."""
     from paper_2603_06588_b200 import binding
+    torch.cuda.set_device(0)
+    ctx = Ctx(binding.HookAttn(0), "cuda:0", load_peaks())
+    name = args.workload
+    if name in ("cfg5_prefill", "cfg5_decode"):
+        sess = Session(ctx, binding, steps=128)
+        case = sess.prefill if name == "cfg5_prefill" else sess.decodes[64]
+        w = session_part(sess, name)
+    else:
+        w = build(ctx, name, binding)
+        case = w.get("case")
+    flush = None
+    if case is not None and algorithmic_work(case)[0] < 256e6:       # inputs do not exceed L2: flush between steps
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda:0")
+    sampler = ClockSampler(0)
+    sampler.start()
+    windows = {}
+    if flush is None:
+        spb = max(1, args.steps // 5) if args.steps else 0
+        entry, _ = measure_entry(ctx, name, w, max(args.warmup, 3), windows, steps_per_block=spb)
+    else:
+        # one step per timed block, an L2 flush (outside the events) before each
+        for _ in range(max(args.warmup, 3)):
+            w["hooked"]()
+            w["plain"]()
+        th, tp = [], []
+        e0, e1 = _event_pair()
+        w0 = time.time()
+        for _ in range(max(args.steps, 5)):
+            for fn, acc in ((w["plain"], tp), (w["hooked"], th)):
+                flush.zero_()
+                e0.record()
+                fn()
+                e1.record()
+                e1.synchronize()
+                acc.append(e0.elapsed_time(e1) / 1e3)
+        windows[name] = (w0, time.time())
+        per_step = statistics.median(th)
+        entry = {"workload": WORKLOADS[name], "tokens_per_step": w["tokens"], "tokens_per_s": w["tokens"] / per_step}
+        entry.update(stats(th))
+        entry.update({"steps_per_block": 1, "ms_per_step_hooks_off": statistics.median(tp) * 1e3,
+                      "hook_overhead": statistics.median(h / p for h, p in zip(th, tp)) - 1.0,
+                      "roofline": roofline(w["bound"], w["work"], per_step, ctx.peaks, w["kernel"], 0.0, DRAM_TRAFFIC.get(name)),
+                      "gpu_launches_per_step": w["launches"]})
+    sampler.stop()
+    line = {"metric": METRIC, "value": entry["tokens_per_s"], "unit": UNIT, "n_gpus": 1,
+            "steps": entry["steps_per_block"] * entry["blocks"], "warmup": max(args.warmup, 3), "ms_per_step": entry["ms_per_step"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{name}: {WORKLOADS[name]}",
+                       "l2": "inputs larger than L2" if flush is None else "L2 flushed between iterations (256 MB write)"},
+            "roofline": entry["roofline"], "hook_overhead": entry["hook_overhead"],
+            "ms_per_step_hooks_off": entry["ms_per_step_hooks_off"], "ms_min": entry["ms_min"], "ms_max": entry["ms_max"],
+            "e2e": None, "gpu_launches": entry["gpu_launches_per_step"] * entry["steps_per_block"] * entry["blocks"],
+            "clocks": sampler.window(*windows[name])}
+    print(json.dumps(line))
+
+
+def session_part(sess, name):
+    """The prefill call or one decode step of a session as a workload of its own."""
+    if name == "cfg5_prefill":
+        return {"hooked": sess.pf_h.run, "plain": sess.pf_p.run, "tokens": sess.prefill.total_q, "bound": "tensor",
+                "work": sess.flops_pf, "kernel": "prefill_tc_kernel", "launches": 1}
+    mid = len(sess.decodes) // 2
+    return {"hooked": sess.dec_h[mid].run, "plain": sess.dec_p[mid].run, "tokens": sess.decodes[mid].total_q, "bound": "hbm",
+            "work": algorithmic_work(sess.decodes[mid])[0], "kernel": decode_kernel_name(sess.decodes[mid]), "launches": 2}
+
+
+# ------------------------------------------------------------------------------------------------
+def run_headline(args):
+    from paper_2603_06588_b200 import binding, replicas
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -480,6 +612,7 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
     if dist:
         import torch.distributed as td
         td.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -489,180 +622,146 @@ def main():
             td.barrier()
         torch.cuda.synchronize()
 
-    case = make_workload(args.workload)
-    eng = binding.HookAttn(local)
-    kw = binding.case_to_device(case, f"cuda:{local}")
-    kw_off = binding.case_to_device(case.without_hooks(), f"cuda:{local}")
-    for k in ("q", "k_cache", "v_cache", "block_table", "seq_lens", "cu_q_lens"):
-        if k in kw:
-            kw_off[k] = kw[k]                       # same device tensors, hooks disabled
-    status = torch.zeros(1, dtype=torch.int32, device=f"cuda:{local}")
-    plan_hook = eng.plan(case.is_decode, status=status, **kw)      # marshals once, allocates outputs
-    plan_off = eng.plan(case.is_decode, **kw_off)
-    plan_hook.run()
-    plan_off.run()
-    out, mass = plan_hook.out, plan_hook.span_mass
-    torch.cuda.synchronize()
-    if int(status.item()) != 0:
-        raise SystemExit(f"device status {binding.strerror(int(status.item()))}")
-    launches_per_step = 2 if case.is_decode else 1
-
-    def timed(n, plan):
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        ev0.record()
-        for _ in range(n):
-            plan.run()
-        ev1.record()
-        barrier()
-        return ev0.elapsed_time(ev1) / 1e3
-
-    alg_bytes, alg_flops = algorithmic_work(case)
-    working_set_mb = alg_bytes / 1e6
-    flush = None
-    if working_set_mb < 256:                         # inputs do not exceed L2: flush between iterations
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device=f"cuda:{local}")
-
-    def timed_flushed(n, plan):
-        tot = 0.0
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
-        for _ in range(n):
-            flush.zero_()
-            ev0.record()
-            plan.run()
-            ev1.record()
-            ev1.synchronize()
-            tot += ev0.elapsed_time(ev1) / 1e3
-        barrier()
-        return tot
-
-    run_timed = timed if flush is None else timed_flushed
-    hooked, plain = plan_hook, plan_off
-
-    run_timed(args.warmup, hooked)
+    peaks = load_peaks()
+    ctx = Ctx(binding.HookAttn(local), dev, peaks)
+    warmup = max(args.warmup, 3)
+    blocks = 5
+    spb = max(1, math.ceil(args.steps / blocks))              # the timed steps, in five blocks
+    steps = spb * blocks
     sampler = ClockSampler(local)
     sampler.start()
-    t_hook = run_timed(args.steps, hooked)
-    clocks_timed = sampler.stop()
+    windows, table = {}, {}
 
-    # hook overhead: same kernels with hooks disabled, interleaved with hooked passes
-    sampler2 = ClockSampler(local)
-    sampler2.start()
-    reps = 7
-    n_ov = max(20, min(args.steps, 200))
-    th, tp = [], []
-    for _ in range(reps):
-        tp.append(run_timed(n_ov, plain) / n_ov)
-        th.append(run_timed(n_ov, hooked) / n_ov)
-    # median of the ratios of neighbouring (hooked, plain) passes: clock drift under the power cap
-    # moves both members of a pair alike
-    overhead = statistics.median(h / p for h, p in zip(th, tp)) - 1.0
+    # ---- the headline: the long-context session, hooks on and off ----
+    sess = Session(ctx, binding, probed=64)
+    head, th = measure_entry(ctx, HEADLINE, sess.entry(), warmup, windows, steps_per_block=spb, blocks=blocks, sync=barrier)
+    barrier()
+    t_step = sum(th) / len(th)                                 # mean over exactly `steps` timed steps
 
-    # end to end through the public call with host buffers: the step's inputs (queries, tables,
-    # lengths, spans) come from pinned host memory and the results go back to the host every step;
-    # the KV cache is state that stays resident on the device, like it does while serving.
-    # The step's inputs are packed into one pinned host buffer and one device buffer (256-byte aligned
-    # views), the results into one device buffer and one pinned host buffer: one copy each way.
-    dev_str = f"cuda:{local}"
-
-    def pack(tensors, device, pin=False):
-        offs, total = {}, 0
-        for k, t in tensors.items():
-            offs[k] = total
-            total += (t.numel() * t.element_size() + 255) // 256 * 256
-        buf = torch.empty(total, dtype=torch.uint8, device=device)
-        if pin:
-            buf = buf.pin_memory()
-        views = {k: buf[offs[k]:offs[k] + t.numel() * t.element_size()].view(t.dtype).view(t.shape) for k, t in tensors.items()}
-        return buf, views
-
-    step_in = {k: kw[k] for k in ("q", "block_table", "seq_lens", "cu_q_lens", "spans") if k in kw}
-    host_in_buf, host_in = pack(step_in, "cpu", pin=True)
-    for k, t in step_in.items():
-        host_in[k].copy_(t)
-    dev_in_buf, dev_in = pack(step_in, dev_str)
-    step_out = {"out": out} if mass is None else {"out": out, "mass": mass}
-    dev_out_buf, dev_out = pack(step_out, dev_str)
-    host_out_buf, _host_out = pack(step_out, "cpu", pin=True)
-    e2e_kw = dict(kw)
-    e2e_kw.update(dev_in)
-    plan_e2e = eng.plan(case.is_decode, out=dev_out["out"], span_mass=dev_out.get("mass"), **e2e_kw)
-    h2d = sum(t.numel() * t.element_size() for t in step_in.values())
-    d2h = sum(t.numel() * t.element_size() for t in step_out.values())
+    # ---- end to end: the step's inputs from pinned host memory, its results back to the host ----
+    pf, dec0 = sess.pf_h, sess.dec_h[0]
+    kw_pf = binding.case_to_device(sess.prefill, dev)         # the session's own device tensors
+    q_pf = kw_pf["q"]
+    pf_small = {k: kw_pf[k].clone() for k in ("block_table", "seq_lens", "cu_q_lens", "spans")}
+    dec_q = binding.case_to_device(sess.decodes[0], dev)["q"]
+    host_q_pf = torch.empty(q_pf.shape, dtype=torch.bfloat16).pin_memory()
+    host_q_pf.copy_(q_pf)
+    host_small = {k: v.cpu().pin_memory() for k, v in pf_small.items()}
+    host_dec_q = dec_q.cpu().pin_memory()
+    host_dec_len = [L.cpu().pin_memory() for L in sess.dec_len]
+    host_out = {"out_pf": torch.empty(pf.out.shape, dtype=torch.bfloat16).pin_memory(),
+                "mass_pf": torch.empty(pf.span_mass.shape, dtype=torch.float32).pin_memory(),
+                "out_dec": torch.empty((len(sess.decodes),) + tuple(dec0.out.shape), dtype=torch.bfloat16).pin_memory(),
+                "mass_dec": torch.empty((len(sess.decodes),) + tuple(dec0.span_mass.shape), dtype=torch.float32).pin_memory()}
+    # the prefill call of the e2e step reads tables, lengths and spans from buffers that the step fills from the host
+    e2e_pf = ctx.eng.plan(False, status=ctx.status, out=pf.out, span_mass=pf.span_mass, **dict(kw_pf, **pf_small))
 
     def e2e_step():
-        dev_in_buf.copy_(host_in_buf, non_blocking=True)
-        plan_e2e.run()
-        host_out_buf.copy_(dev_out_buf, non_blocking=True)
+        q_pf.copy_(host_q_pf, non_blocking=True)
+        for k, v in host_small.items():
+            pf_small[k].copy_(v, non_blocking=True)
+        e2e_pf.run()
+        host_out["out_pf"].copy_(pf.out, non_blocking=True)
+        host_out["mass_pf"].copy_(pf.span_mass, non_blocking=True)
+        for t, plan in enumerate(sess.dec_h):
+            dec_q.copy_(host_dec_q, non_blocking=True)
+            sess.dec_len[t].copy_(host_dec_len[t], non_blocking=True)
+            plan.run()
+            host_out["out_dec"][t].copy_(dec0.out, non_blocking=True)
+            host_out["mass_dec"][t].copy_(dec0.span_mass, non_blocking=True)
         torch.cuda.current_stream().synchronize()
 
-    n_e2e = max(10, min(args.steps, 500))
-    for _ in range(3):
-        e2e_step()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h2d = (host_q_pf.numel() * 2 + sum(v.numel() * v.element_size() for v in host_small.values())
+           + len(sess.decodes) * (host_dec_q.numel() * 2 + host_dec_len[0].numel() * 4))
+    d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+    e2e_step()
     barrier()
-    ev0.record()
+    e0, e1 = _event_pair()
+    n_e2e = 3
+    e0.record()
     for _ in range(n_e2e):
         e2e_step()
-    ev1.record()
+    e1.record()
     barrier()
-    t_e2e = ev0.elapsed_time(ev1) / 1e3 / n_e2e
-    clocks_all = sampler2.stop()
+    t_e2e = e0.elapsed_time(e1) / 1e3 / n_e2e
+    del host_q_pf, host_out, e2e_pf
 
-    from paper_2603_06588_b200 import replicas
-    t_hook, t_e2e = replicas.max_over_ranks([t_hook, t_e2e], torch.device("cuda", local))
+    t_step, t_e2e = replicas.max_over_ranks([t_step, t_e2e], torch.device("cuda", local))
+
+    # ---- every other named workload (one GPU only: they are single-GPU measurements) ----
+    if not dist and not args.headline_only:
+        table["cfg5_prefill"], _ = measure_entry(ctx, "cfg5_prefill", session_part(sess, "cfg5_prefill"), warmup, windows)
+        table["cfg5_decode"], _ = measure_entry(ctx, "cfg5_decode", session_part(sess, "cfg5_decode"), warmup, windows)
+        del sess
+        torch.cuda.empty_cache()
+        s16 = Session(ctx, binding, probed=16)
+        table["cfg5_16of64"], _ = measure_entry(ctx, "cfg5_16of64", s16.entry(), warmup, windows)
+        del s16
+        torch.cuda.empty_cache()
+        for name in ("cfg2_decode", "cfg4_decode", "cfg4_prefill", "cfg4_mixed", "cfg3_prefill_32layers"):
+            w = build(ctx, name, binding)
+            table[name], _ = measure_entry(ctx, name, w, warmup, windows)
+            del w
+            torch.cuda.empty_cache()
+    sampler.stop()
 
     if rank == 0:
-        peaks = load_peaks()
-        per_step = t_hook / args.steps
-        tokens = case.total_q
-        bound = "hbm" if case.is_decode else "tensor"
-        if bound == "hbm":
-            achieved = alg_bytes / per_step / 1e9
-            peak, unit = peaks["hbm_gbs"], "GB/s"
-        else:
-            achieved = alg_flops / per_step / 1e12
-            peak, unit = (peaks["bf16_tflops"] if t_hook < 2.0 else peaks["bf16_tflops_sustained"]), "TFLOP/s"
-        clocks = clocks_timed if clocks_timed["samples"] >= 3 else clocks_all
+        for name, e in table.items():
+            e["clocks"] = sampler.window(*windows[name])
+        roof = head["roofline"]
         line = {
-            "metric": METRIC, "value": replicas.replica_throughput(tokens, per_step, world), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"{args.workload}: {WORKLOADS[args.workload]}",
-                       "l2": ("inputs larger than L2 (%.0f MB per step)" % working_set_mb) if flush is None
-                       else "L2 flushed between iterations (256 MB write)",
-                       "replicas": world, "kv_cache": "resident in HBM (state, not a per-step input)"},
-            "roofline": {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
-                         "traffic": DRAM_TRAFFIC.get(args.workload), "peak_source": f"of {peaks['source']}",
-                         "kernel": (("decode_stream_kernel" if case.num_seqs * case.num_kv_heads < 296 else "decode_splitk_kernel")
-                                    + " (+ decode_merge_kernel; duration = whole step, conservative)")
-                         if case.is_decode else "prefill_tc_kernel (one launch per step)",
-                         "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
-                         "frac_of_datasheet": achieved / (8000.0 if bound == "hbm" else 2250.0)},
-            "hook_overhead": overhead,
-            "ms_per_step_hooks_off": statistics.median(tp) * 1e3,
-            "e2e": {"value": replicas.replica_throughput(tokens, t_e2e, world), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "ms_per_step": t_e2e * 1e3},
-            "gpu_launches": launches_per_step * args.steps,
-            "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
-                       "samples": clocks["samples"], "sm_mhz_min": clocks["sm_mhz_min"], "power_w": clocks["power_w"]},
+            "metric": METRIC, "value": replicas.replica_throughput(head["tokens_per_step"], t_step, world), "unit": UNIT,
+            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": t_step * 1e3,
+            "ms_per_step_median_of_blocks": head["ms_per_step"], "ms_min": head["ms_min"], "ms_max": head["ms_max"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{HEADLINE}: {WORKLOADS[HEADLINE]}",
+                       "l2": "inputs larger than L2 (2.7 GB of q/K/V per prefill call, 0.54 GB of K/V per decode step)",
+                       "replicas": world, "kv_cache": "resident in HBM (state, not a per-step input)",
+                       "inputs": "drawn on the device by a seeded generator (same recipe as the CPU-drawn test inputs)"},
+            "roofline": roof, "hook_overhead": head["hook_overhead"], "ms_per_step_hooks_off": head["ms_per_step_hooks_off"],
+            "prefill_ms": head["prefill_ms"], "decode_ms_per_step": head["decode_ms_per_step"], "decode_gbs": head["decode_gbs"],
+            "e2e": {"value": replicas.replica_throughput(head["tokens_per_step"], t_e2e, world), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e * 1e3, "steps": n_e2e},
+            "gpu_launches": head["gpu_launches_per_step"] * steps,
+            "clocks": sampler.window(*windows[HEADLINE]),
+            "workloads": table,
         }
         if not args.no_cpu_baseline:
-            from oracle import oracle
-            rows, desc, scale_tokens = oracle_sample(case, budget_s=2.0)
-            oracle.run(case, rows=rows[: max(1, len(rows) // 8)])
-            t0 = time.perf_counter()
-            reps_cpu = 3
-            for _ in range(reps_cpu):
-                oracle.run(case, rows=rows)
-            dt = (time.perf_counter() - t0) / reps_cpu
-            line["cpu_baseline"] = {"value": scale_tokens / dt, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-                                    "sample": desc, "seconds_per_pass": dt}
+            cases = inputs.config5_session(device=dev)
+            val, dt, desc, cores = run_oracle_sample(cases, budget_s=8.0, reps=2)
+            line["cpu_baseline"] = dict({"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                                         "seconds_per_pass": dt}, **host_cores())
         print(json.dumps(line))
     if dist:
         td.barrier()
         td.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=None, help="time one named workload by itself instead of the headline + table")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-budget", type=float, default=8.0, help="seconds of CPU time per oracle step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true", help="skip the table of the other workloads")
+    args = ap.parse_args()
+    if args.workload is not None and args.workload not in WORKLOADS:
+        raise SystemExit(f"unknown workload {args.workload}; choose from {sorted(WORKLOADS)}")
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    from paper_2603_06588_b200.csrc import build as cuda_build
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        cuda_build.build()      # no-op when the in-tree library is up to date
+    if args.workload in ("steer_residual", "capture_qk"):
+        run_extra(args)
+    elif args.workload is not None and args.workload != HEADLINE:
+        run_one(args)
+    else:
+        run_headline(args)
 
 
 if __name__ == "__main__":

@@ -17,8 +17,8 @@
  *       attention head after the softmax normalisation and before the single rounding of
  *       the output to bf16.
  *
- * Probing never changes `out` ("keeping the model generation intact", Section 1): with and
- * without probes the output bits are identical.  No attention matrix is materialised and no
+ * Probing never changes `out` (Section 1 requires that passive programming leaves the model's
+ * generation as it is): with and without probes the output bits are identical.  No attention matrix is materialised and no
  * query/key tensor leaves the GPU; span masses are carried as extra online-softmax
  * accumulators.
  *
@@ -34,8 +34,10 @@
  * caller's stream, never synchronise, and never allocate device memory.  Return codes are
  * synchronous and cover argument validation and launch errors; faults the device detects
  * (a block-table entry outside [0, num_blocks), a sequence longer than its table, more rows
- * than keys) are reported through the optional `status` word, the affected rows are written
- * as zeros, and no out-of-range address is dereferenced.
+ * than keys, a sequence longer than `max_seq_len`) are reported through the optional `status`
+ * word, the affected rows of `out` and `span_mass` are written as zeros, and no out-of-range
+ * address is dereferenced.  Every entry point that launches work returns
+ * HOOK_ATTN_ERR_INVALID_ARG unless the handle's device is the current device.
  *
  * Supported: head_dim in {64, 128}; page_size = 16; num_q_heads % num_kv_heads == 0 with a
  * group size <= 8; num_q_heads <= 64; num_spans <= 8; strides multiples of 8 elements and
@@ -51,7 +53,8 @@
 extern "C" {
 #endif
 
-typedef struct hook_attn_handle hook_attn_handle; /* per-device state: SM count, cached descriptors */
+typedef struct hook_attn_handle hook_attn_handle; /* per-device state: SM count, cache of the prefill
+                                                     kernel's TMA descriptors (keyed by pointer, shape, strides) */
 
 enum {
     HOOK_ATTN_OK = 0,
@@ -82,7 +85,11 @@ typedef struct {
     int32_t num_spans;           /* S spans per sequence (0 = no probe) */
     int32_t probe_rows;          /* HOOK_PROBE_ROWS_*; ignored by decode (always LAST) */
     float   scale;               /* softmax scale; <= 0 selects 1/sqrt(head_dim) */
-    int32_t reserved0;
+    int32_t max_seq_len;         /* optional host-side bound on seq_lens (0 = unknown, then
+                                    max_blocks_per_seq * page_size).  Block tables are often padded to
+                                    the model's maximum length; with the bound, decode cuts its work and
+                                    sizes its workspace for the lengths the batch really has.  A sequence
+                                    longer than the bound is a device-detected fault (status, zeros). */
 
     /* ---- device tensors ---- */
     const void*    q;            /* bf16 [total_q][Hq][D], contiguous */
@@ -100,8 +107,10 @@ typedef struct {
     void*          out;          /* bf16 [total_q][Hq][D] */
     float*         span_mass;    /* fp32 [rows][P][S]; rows = total_q (ALL) or num_seqs (LAST, decode);
                                     P = number of nonzero head_mask entries; the slot of a probed head is
-                                    its rank among the probed heads in ascending head order */
-    void*          workspace;    /* scratch of at least hook_attn_workspace_bytes(); 256-byte aligned */
+                                    its rank among the probed heads in ascending head order.  In LAST mode
+                                    a sequence without rows in the call gets zeros */
+    void*          workspace;    /* scratch of at least hook_attn_workspace_bytes(); 256-byte aligned
+                                    (checked: HOOK_ATTN_ERR_WORKSPACE otherwise) */
     size_t         workspace_bytes;
     int32_t*       status;       /* optional: one int32, set to a negative HOOK_ATTN_ERR_* code by the
                                     device on a detected fault; the caller zeroes it beforehand */
@@ -117,7 +126,8 @@ typedef struct {
 int hook_attn_create(hook_attn_handle** handle, int device);
 int hook_attn_destroy(hook_attn_handle* handle);
 
-/* Bytes of scratch the call described by `p` needs (only the shape fields are read).
+/* Bytes of scratch the call described by `p` needs (only the shape fields and max_seq_len are read;
+ * pass the same max_seq_len to the call).
  * is_decode != 0 sizes hook_attn_decode, 0 sizes hook_attn_prefill.  Returns 0 when the call needs
  * no scratch or when the shapes are invalid. */
 size_t hook_attn_workspace_bytes(const hook_attn_params* p, int is_decode);
@@ -126,10 +136,14 @@ size_t hook_attn_workspace_bytes(const hook_attn_params* p, int is_decode);
  * (Section 2.2 recompute + Section 2 steering, fused into the attention forward.) */
 int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
 
-/* Decode: exactly one query row per sequence (total_q == num_seqs, cu_q_lens ignored).  The keys
- * of all sequences are dealt out in equal shares to a fixed number of workers; each share is
- * reduced independently and the pieces of a sequence are merged in a fixed order, so results are
- * bit-identical from run to run.  span_mass has one row per sequence. */
+/* Decode: exactly one query row per sequence (total_q == num_seqs, cu_q_lens ignored).  The keys of a
+ * (sequence, KV head) unit are cut into pieces that are reduced independently and then merged.  The
+ * cut is chosen from the host-known shape of the batch: with many units (num_seqs * num_kv_heads >=
+ * 296) every sequence is cut into chunks of a fixed length (a power of two in 256..2048 keys, from
+ * num_seqs, num_kv_heads and the length bound); with fewer, the pages of all units form one list
+ * that is dealt out in equal shares to a fixed number of worker warps.  Either way the pieces of a
+ * unit are merged in a fixed order, so results are bit-identical from run to run.  span_mass has one
+ * row per sequence. */
 int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
 
 /* Decode for callers that can neither allocate device memory nor hand over scratch.

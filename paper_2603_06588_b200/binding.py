@@ -42,7 +42,7 @@ class HookAttnParams(ctypes.Structure):
         ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
         ("num_blocks", ctypes.c_int32), ("max_blocks_per_seq", ctypes.c_int32),
         ("num_spans", ctypes.c_int32), ("probe_rows", ctypes.c_int32),
-        ("scale", ctypes.c_float), ("reserved0", ctypes.c_int32),
+        ("scale", ctypes.c_float), ("max_seq_len", ctypes.c_int32),
         ("q", ctypes.c_void_p), ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
         ("kv_block_stride", ctypes.c_int64), ("kv_token_stride", ctypes.c_int64),
         ("kv_head_stride", ctypes.c_int64),
@@ -112,7 +112,7 @@ def _dptr(t: Optional[torch.Tensor]) -> Optional[int]:
 def make_params(*, q, k_cache, v_cache, block_table, seq_lens, cu_q_lens=None, spans=None,
                 head_mask=None, alpha=None, steer_vec=None, scale: float = 0.0,
                 probe_rows: int = HOOK_PROBE_ROWS_ALL, out=None, span_mass=None, workspace=None,
-                status=None) -> Tuple[HookAttnParams, list]:
+                status=None, max_seq_len: int = 0) -> Tuple[HookAttnParams, list]:
     """Marshal tensors into a ``hook_attn_params``.  ``head_mask`` / ``alpha`` are HOST tensors
     (uint8 / float32); everything else lives on the device.  Returns the struct and a list of
     objects that must stay alive until the call has been issued."""
@@ -130,6 +130,7 @@ def make_params(*, q, k_cache, v_cache, block_table, seq_lens, cu_q_lens=None, s
     p.num_spans = 0 if spans is None else int(spans.shape[1])
     p.probe_rows = int(probe_rows)
     p.scale = float(scale)
+    p.max_seq_len = int(max_seq_len)
     p.q, p.k_cache, p.v_cache = q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr()
     p.kv_block_stride, p.kv_token_stride, p.kv_head_stride = (int(k_cache.stride(0)),
                                                                int(k_cache.stride(1)),
@@ -237,7 +238,7 @@ class HookAttn:
 
     def hook_capture_qk(self, is_decode: bool, *, q, k_cache, v_cache, block_table, seq_lens, cu_q_lens=None,
                         head_mask=None, probe_rows=HOOK_PROBE_ROWS_ALL, status=None, stream=None,
-                        q_out=None, k_out=None, cu_k_lens=None, **_ignored):
+                        q_out=None, k_out=None, cu_k_lens=None, max_seq_len: int = 0, **_ignored):
         """Raw q/k capture of the probed heads.  Returns ``(q_out [rows, P, D], k_out [sum L, P, D], cu_k_lens)``.
         The three outputs are allocated (and the prefix sums computed, with one host sync for the total)
         unless the caller passes them."""
@@ -254,7 +255,8 @@ class HookAttn:
         if k_out is None:
             k_out = torch.zeros((int(cu_k[-1].item()), nprobed, d), dtype=torch.bfloat16, device=q.device)
         p, keep = make_params(q=q, k_cache=k_cache, v_cache=v_cache, block_table=block_table, seq_lens=seq_lens,
-                              cu_q_lens=cu_q_lens, head_mask=head_mask, probe_rows=probe_rows, status=status)
+                              cu_q_lens=cu_q_lens, head_mask=head_mask, probe_rows=probe_rows, status=status,
+                              max_seq_len=max_seq_len)
         rc = int(self._lib.hook_capture_qk(self._h, ctypes.byref(p), int(bool(is_decode)), q_out.data_ptr(),
                                            k_out.data_ptr(), cu_k.data_ptr(), self._stream(stream)))
         del keep
@@ -265,7 +267,8 @@ class HookAttn:
     # -- convenience ---------------------------------------------------------------------
     def plan(self, is_decode: bool, *, q, k_cache, v_cache, block_table, seq_lens, cu_q_lens=None,
              spans=None, head_mask=None, alpha=None, steer_vec=None, scale=0.0,
-             probe_rows=HOOK_PROBE_ROWS_ALL, out=None, span_mass=None, status=None) -> "HookAttnPlan":
+             probe_rows=HOOK_PROBE_ROWS_ALL, out=None, span_mass=None, status=None,
+             max_seq_len: int = 0) -> "HookAttnPlan":
         """Marshal the arguments once (allocating `out`, `span_mass` and scratch when they are not
         given); the returned plan re-issues the same call with one C call per step."""
         total_q, hq, d = q.shape
@@ -279,7 +282,8 @@ class HookAttn:
         p, keep = make_params(q=q, k_cache=k_cache, v_cache=v_cache, block_table=block_table,
                               seq_lens=seq_lens, cu_q_lens=cu_q_lens, spans=spans,
                               head_mask=head_mask, alpha=alpha, steer_vec=steer_vec, scale=scale,
-                              probe_rows=probe_rows, out=out, span_mass=span_mass, status=status)
+                              probe_rows=probe_rows, out=out, span_mass=span_mass, status=status,
+                              max_seq_len=max_seq_len)
         nbytes = self.workspace_bytes(p, is_decode)
         ws = None
         if nbytes:

@@ -10,8 +10,8 @@
 namespace hook_attn {
 // decode.cu
 cudaError_t configure_decode();
-cudaError_t launch_decode(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st);
-size_t decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim, int max_blocks);
+cudaError_t launch_decode(const KernelArgs& a, const HeadCfg& hc, int head_dim, int num_sms, cudaStream_t st);
+size_t decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim, int max_keys);
 // prefill_mma.cu
 cudaError_t configure_prefill_mma();
 cudaError_t launch_prefill_mma(const KernelArgs& a, const HeadCfg& hc, int head_dim, cudaStream_t st);
@@ -19,7 +19,9 @@ int prefill_mma_tiles_upper_bound(int total_q, int num_seqs);
 // prefill_tc.cu
 cudaError_t configure_prefill_tc();
 bool prefill_tc_supported(const KernelArgs& a, int head_dim);
-cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, cudaStream_t st);
+cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, void* tmap_cache, int num_sms, cudaStream_t st);
+void* tmap_cache_create();
+void tmap_cache_destroy(void* cache);
 cudaError_t launch_wait_selftest(int32_t* status, uint64_t limit_ns, uint64_t* waited_ns, cudaStream_t st);
 // extras.cu
 cudaError_t launch_score(const float* mass, float* scores, int rows, int P, int S, int mode, cudaStream_t st);
@@ -36,6 +38,7 @@ struct hook_attn_handle {
     int num_sms;
     int cc_major, cc_minor;
     bool prefer_tc;   // head_dim-128 prefill goes to the tcgen05 kernel (HOOK_ATTN_PREFILL_KERNEL=mma turns it off)
+    void* tmap_cache; // TMA descriptors of the prefill kernel, keyed by base pointer, shape and strides
 };
 
 namespace {
@@ -44,7 +47,7 @@ int validate_common(const hook_attn_params* p, bool decode)
 {
     if (!p) return HOOK_ATTN_ERR_INVALID_ARG;
     if (p->num_seqs < 0 || p->total_q < 0 || p->num_q_heads <= 0 || p->num_kv_heads <= 0 || p->head_dim <= 0 ||
-        p->page_size <= 0 || p->num_blocks < 0 || p->max_blocks_per_seq < 0 || p->num_spans < 0)
+        p->page_size <= 0 || p->num_blocks < 0 || p->max_blocks_per_seq < 0 || p->num_spans < 0 || p->max_seq_len < 0)
         return HOOK_ATTN_ERR_INVALID_ARG;
     if (p->num_q_heads % p->num_kv_heads != 0) return HOOK_ATTN_ERR_INVALID_ARG;
     if (decode && p->total_q != p->num_seqs) return HOOK_ATTN_ERR_INVALID_ARG;
@@ -59,6 +62,25 @@ int validate_common(const hook_attn_params* p, bool decode)
 }
 
 bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+
+// Longest sequence the call may hold: the caller's hint when given, never more than the table can address.
+int max_keys_of(const hook_attn_params* p)
+{
+    long long cap = (long long)p->max_blocks_per_seq * p->page_size;
+    if (cap > 0x7fffffffLL) cap = 0x7fffffffLL;
+    if (p->max_seq_len > 0 && p->max_seq_len < cap) cap = p->max_seq_len;
+    return (int)cap;
+}
+
+// Calls that launch need the handle's device to be the current one: the launch goes to the current
+// device, and the kernels' shared-memory opt-in was made on the handle's.
+int check_handle(const hook_attn_handle* handle)
+{
+    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess) { (void)cudaGetLastError(); return HOOK_ATTN_ERR_CUDA; }
+    return current == handle->device ? HOOK_ATTN_OK : HOOK_ATTN_ERR_INVALID_ARG;
+}
 
 // Fills the kernel arguments; returns a HOOK_ATTN_* code.
 int prepare(const hook_attn_params* p, bool decode, KernelArgs& a, HeadCfg& hc)
@@ -103,6 +125,7 @@ int prepare(const hook_attn_params* p, bool decode, KernelArgs& a, HeadCfg& hc)
     a.num_seqs = p->num_seqs; a.total_q = p->total_q; a.Hq = p->num_q_heads; a.Hkv = p->num_kv_heads;
     a.G = p->num_q_heads / p->num_kv_heads;
     a.num_blocks = p->num_blocks; a.max_blocks = p->max_blocks_per_seq;
+    a.max_keys = max_keys_of(p);
     a.S = any_probe ? p->num_spans : 0; a.P = probed; a.probe_rows = p->probe_rows;
     const float scale = (p->scale > 0.f) ? p->scale : 1.0f / sqrtf((float)p->head_dim);
     a.scale_log2 = scale * 1.4426950408889634f;
@@ -141,12 +164,14 @@ int hook_attn_create(hook_attn_handle** handle, int device)
     h->cc_minor = prop.minor;
     const char* pk = getenv("HOOK_ATTN_PREFILL_KERNEL");
     h->prefer_tc = !(pk && strcmp(pk, "mma") == 0);
+    h->tmap_cache = tmap_cache_create();
     *handle = h;
     return HOOK_ATTN_OK;
 }
 
 int hook_attn_destroy(hook_attn_handle* handle)
 {
+    if (handle) tmap_cache_destroy(handle->tmap_cache);
     delete handle;
     return HOOK_ATTN_OK;
 }
@@ -156,7 +181,7 @@ size_t hook_attn_workspace_bytes(const hook_attn_params* p, int is_decode)
     if (validate_common(p, is_decode != 0) != HOOK_ATTN_OK) return 0;
     if (!is_decode) return 0;
     const int G = p->num_q_heads / p->num_kv_heads;
-    return decode_workspace_bytes(p->num_seqs, p->num_kv_heads, G, p->head_dim, p->max_blocks_per_seq);
+    return decode_workspace_bytes(p->num_seqs, p->num_kv_heads, G, p->head_dim, max_keys_of(p));
 }
 
 int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream)
@@ -165,11 +190,11 @@ int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void*
     HeadCfg hc;
     int rc = prepare(p, false, a, hc);     // argument errors are reported before anything else
     if (rc != HOOK_ATTN_OK) return rc;
-    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    if ((rc = check_handle(handle)) != HOOK_ATTN_OK) return rc;
     if (p->num_seqs == 0 || p->total_q == 0) return HOOK_ATTN_OK;
     cudaError_t e;
     if (handle->prefer_tc && prefill_tc_supported(a, p->head_dim)) {
-        e = launch_prefill_tc(a, hc, static_cast<cudaStream_t>(cuda_stream));
+        e = launch_prefill_tc(a, hc, handle->tmap_cache, handle->num_sms, static_cast<cudaStream_t>(cuda_stream));
     } else {
         a.total_tiles = prefill_mma_tiles_upper_bound(p->total_q, p->num_seqs);
         e = launch_prefill_mma(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
@@ -185,11 +210,11 @@ int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* 
     if (rc != HOOK_ATTN_OK) return rc;
     if (p->num_seqs > 0 && p->max_blocks_per_seq == 0) return HOOK_ATTN_ERR_INVALID_ARG;
     if (p->num_seqs == 0) return handle ? HOOK_ATTN_OK : HOOK_ATTN_ERR_INVALID_ARG;
-    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, p->max_blocks_per_seq);
+    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, a.max_keys);
     if (!p->workspace || p->workspace_bytes < need) return HOOK_ATTN_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(p->workspace) & 15u) return HOOK_ATTN_ERR_WORKSPACE;
-    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
-    cudaError_t e = launch_decode(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
+    if (reinterpret_cast<uintptr_t>(p->workspace) & 255u) return HOOK_ATTN_ERR_WORKSPACE;
+    if ((rc = check_handle(handle)) != HOOK_ATTN_OK) return rc;
+    cudaError_t e = launch_decode(a, hc, p->head_dim, handle->num_sms, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
 }
 
@@ -238,18 +263,15 @@ int hook_attn_decode_static_scratch(hook_attn_handle* handle, const hook_attn_pa
     if (rc != HOOK_ATTN_OK) return rc;
     if (p->num_seqs > 0 && p->max_blocks_per_seq == 0) return HOOK_ATTN_ERR_INVALID_ARG;
     if (p->num_seqs == 0) return handle ? HOOK_ATTN_OK : HOOK_ATTN_ERR_INVALID_ARG;
-    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, p->max_blocks_per_seq);
+    const size_t need = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, a.G, p->head_dim, a.max_keys);
     if (need > HOOK_ATTN_STATIC_SCRATCH_BYTES) return HOOK_ATTN_ERR_WORKSPACE;   // batch too large for the fixed array
-    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
-    int current = -1;
-    if (cudaGetDevice(&current) != cudaSuccess) return HOOK_ATTN_ERR_CUDA;
-    if (current != handle->device) return HOOK_ATTN_ERR_INVALID_ARG;             // the handle's device must be current
+    if ((rc = check_handle(handle)) != HOOK_ATTN_OK) return rc;                  // the handle's device must be current
     float* scratch = nullptr;
     rc = static_scratch_address(handle->device, &scratch);
     if (rc != HOOK_ATTN_OK) return rc;
     a.ws = scratch;   // every partial the merge reads is written by the streaming kernel of the same call:
                       // nothing in the array has to start at zero, stale contents are never read
-    cudaError_t e = launch_decode(a, hc, p->head_dim, static_cast<cudaStream_t>(cuda_stream));
+    cudaError_t e = launch_decode(a, hc, p->head_dim, handle->num_sms, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
 }
 
@@ -260,7 +282,8 @@ int hook_attn_score(hook_attn_handle* handle, const float* span_mass, int32_t ro
     if (mode != HOOK_SCORE_MEAN && mode != HOOK_SCORE_SUM_NORMALIZE) return HOOK_ATTN_ERR_INVALID_ARG;
     if (num_spans > kMaxSpans) return HOOK_ATTN_ERR_UNSUPPORTED;
     if (rows > 0 && (!span_mass || !scores)) return HOOK_ATTN_ERR_INVALID_ARG;
-    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    int rc = check_handle(handle);
+    if (rc != HOOK_ATTN_OK) return rc;
     if (rows == 0) return HOOK_ATTN_OK;
     cudaError_t e = launch_score(span_mass, scores, rows, num_probed, num_spans, mode, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
@@ -273,7 +296,8 @@ int hook_steer_residual(hook_attn_handle* handle, void* hidden, const float* ste
     if ((hidden_size & 7) || (row_stride & 7)) return HOOK_ATTN_ERR_UNSUPPORTED;
     if (num_tokens > 0 && (!hidden || !steer_vec)) return HOOK_ATTN_ERR_INVALID_ARG;
     if (!aligned16(hidden) || !aligned16(steer_vec)) return HOOK_ATTN_ERR_UNSUPPORTED;
-    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    int rc = check_handle(handle);
+    if (rc != HOOK_ATTN_OK) return rc;
     if (num_tokens == 0 || alpha == 0.0f) return HOOK_ATTN_OK;   // alpha = 0 leaves every bit in place
     cudaError_t e = launch_steer_residual(static_cast<__nv_bfloat16*>(hidden), steer_vec, alpha, num_tokens, hidden_size,
                                           row_stride, handle->num_sms, static_cast<cudaStream_t>(cuda_stream));
@@ -293,7 +317,7 @@ int hook_capture_qk(hook_attn_handle* handle, const hook_attn_params* p, int is_
     }
     int rc = prepare(p ? &q : nullptr, is_decode != 0, a, hc);
     if (rc != HOOK_ATTN_OK) return rc;
-    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    if ((rc = check_handle(handle)) != HOOK_ATTN_OK) return rc;
     if (p->num_seqs == 0 || p->total_q == 0) return HOOK_ATTN_OK;
     int probed = 0;
     for (int h = 0; h < p->num_q_heads; ++h)
@@ -311,7 +335,8 @@ int hook_attn_selftest_wait_limit(hook_attn_handle* handle, int32_t* status, uin
                                   void* cuda_stream)
 {
     if (!status || limit_ns == 0 || limit_ns > 1000000000ull) return HOOK_ATTN_ERR_INVALID_ARG;
-    if (!handle) return HOOK_ATTN_ERR_INVALID_ARG;
+    int rc = check_handle(handle);
+    if (rc != HOOK_ATTN_OK) return rc;
     cudaError_t e = launch_wait_selftest(status, limit_ns, waited_ns, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
 }

@@ -36,6 +36,8 @@ struct KernelArgs {
     float* ws;
     int32_t* status;
     int32_t num_seqs, total_q, Hq, Hkv, G, num_blocks, max_blocks, S, P, probe_rows;
+    int32_t max_keys;                 // longest sequence the call may hold: the caller's hint, else max_blocks * page
+    int32_t workers;                  // decode, equal shares: warps that share the flat page list
     int32_t chunk;                    // decode, fixed chunks: keys per chunk
     int32_t max_chunks;               // decode, fixed chunks: chunks per sequence the workspace is sized for
     int32_t total_tiles;              // prefill: upper bound on query tiles

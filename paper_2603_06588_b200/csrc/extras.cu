@@ -96,8 +96,8 @@ __global__ void __launch_bounds__(256) capture_k_kernel(const KernelArgs a, cons
     __syncthreads();
     const int s = blockIdx.y;
     const int L = a.seq_lens[s];
-    if (L <= 0 || L > a.max_blocks * kPage) {
-        if (L > a.max_blocks * kPage && threadIdx.x == 0 && blockIdx.x == 0) report(a.status, HOOK_ATTN_ERR_BOUNDS);
+    if (L <= 0 || L > a.max_keys) {
+        if (L > a.max_keys && threadIdx.x == 0 && blockIdx.x == 0) report(a.status, HOOK_ATTN_ERR_BOUNDS);
         return;
     }
     const int t0 = blockIdx.x * 64;
@@ -162,7 +162,7 @@ cudaError_t launch_capture(const KernelArgs& a, const HeadCfg& hc, int head_dim,
 {
     const bool last_only = decode || a.probe_rows == HOOK_PROBE_ROWS_LAST;
     const int out_rows = last_only ? a.num_seqs : a.total_q;
-    const int key_tiles = (a.max_blocks * kPage + 63) / 64;
+    const int key_tiles = (a.max_keys + 63) / 64;
     if (q_out && out_rows > 0) {
         const int64_t total = (int64_t)out_rows * a.P;
         int blocks = (int)((total + 15) / 16);

@@ -42,6 +42,15 @@ __global__ void __launch_bounds__(128) prefill_mma_kernel(const KernelArgs a, co
     const int g = lane >> 2, tq = lane & 3;
     const int kvh = h / a.G;
 
+    // last-token mode: a sequence without rows in this call gets zeros in its span_mass row
+    if (NS > 0 && blockIdx.x == 0 && blockIdx.y == 0 && a.probe_rows == HOOK_PROBE_ROWS_LAST) {
+        const int per = a.P * a.S;
+        for (int sq = warp; sq < a.num_seqs; sq += 4) {
+            if (a.cu_q_lens[sq + 1] - a.cu_q_lens[sq] > 0) continue;
+            for (int i = lane; i < per; i += 32) a.mass[(int64_t)sq * per + i] = 0.f;
+        }
+    }
+
     // locate (sequence, query tile); later tiles of a sequence (more keys) are scheduled first
     int t = blockIdx.x, s = 0, n = 0;
     for (; s < a.num_seqs; ++s) {
@@ -58,11 +67,20 @@ __global__ void __launch_bounds__(128) prefill_mma_kernel(const KernelArgs a, co
     const int slot = (NS > 0) ? hc.slot[h] : -1;
     const bool probe = (NS > 0) && slot >= 0;
 
-    if (n > L || L > a.max_blocks * kPage) {
+    if (n > L || L > a.max_keys) {
         // inconsistent lengths: report, write zeros for this tile, touch nothing else
         if (threadIdx.x == 0) report(a.status, n > L ? HOOK_ATTN_ERR_INVALID_ARG : HOOK_ATTN_ERR_BOUNDS);
         for (int idx = threadIdx.x; idx < rows * HD; idx += 128)
             a.out[((grow0 + idx / HD) * a.Hq + h) * HD + idx % HD] = __float2bfloat16(0.f);
+        if (probe) {
+            const bool last_only = (a.probe_rows == HOOK_PROBE_ROWS_LAST);
+            for (int idx = threadIdx.x; idx < rows * a.S; idx += 128) {
+                const int r = idx / a.S, js = idx % a.S;
+                if (last_only && row0 + r != n - 1) continue;
+                const int64_t mrow = last_only ? (int64_t)s : grow0 + r;
+                a.mass[(mrow * a.P + slot) * a.S + js] = 0.f;
+            }
+        }
         return;
     }
     const int first_pos = L - n + row0;                 // position of the tile's first row

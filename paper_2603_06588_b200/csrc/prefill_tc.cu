@@ -26,9 +26,17 @@
 // rounding to bf16: a key tile inside a span adds the tile's row sum, a tile that straddles a span
 // edge adds a masked row sum, a disjoint tile adds nothing.
 //
-// Every wait on an mbarrier is bounded; when one runs out the CTA reports HOOK_ATTN_ERR_TIMEOUT
-// through the status word, leaves its loops, releases tensor memory and returns.
+// Every wait on an mbarrier is bounded; when one runs out the role raises the CTA's abort flag (every
+// other wait of the CTA polls it and gives up too), the CTA reports HOOK_ATTN_ERR_TIMEOUT through the
+// status word, stamps a launch-wide word so that the CTAs of the same launch that have not started yet
+// return at once, releases tensor memory and returns.
 #include <cuda.h>
+#include <string.h>
+
+#include <atomic>
+#include <mutex>
+#include <utility>
+#include <vector>
 
 #include "common.cuh"
 
@@ -93,14 +101,22 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after `limit_ns` (two seconds unless stated otherwise).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns = 2000000000ull)
+// Bounded wait: gives up after `limit_ns` (two seconds unless stated otherwise), or as soon as another
+// role of the CTA has given up (`abort_flag`, in shared memory).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag = nullptr,
+                                          uint64_t limit_ns = 2000000000ull)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u && global_timer_ns() - t0 > limit_ns) return false;
+        if ((it & 255u) == 255u) {
+            if (abort_flag && *abort_flag) return false;
+            if (global_timer_ns() - t0 > limit_ns) {
+                if (abort_flag) *abort_flag = 1;
+                return false;
+            }
+        }
     }
 }
 
@@ -218,6 +234,16 @@ __host__ __device__ constexpr uint32_t instr_desc(uint32_t b_mn)
     return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// Set by a CTA whose wait ran out: the id of its launch and the time (globaltimer, ns).  CTAs of the same
+// launch that start within the next seconds return at once instead of sitting out waits of their own, so
+// that a wedged launch of thousands of CTAs ends after one wait limit and not after thousands.
+struct LaunchAbort {
+    unsigned long long when_ns;
+    unsigned int launch_id;
+};
+__device__ LaunchAbort g_launch_abort;
+constexpr unsigned long long kAbortWindowNs = 5000000000ull;
+
 struct Barriers {
     uint64_t q_full[2];
     uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
@@ -233,7 +259,7 @@ using namespace tc;
 
 template <int NS>
 __global__ void __launch_bounds__(kThreads, 1)
-prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ CUtensorMap map_q,
+prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const unsigned int launch_id, const __grid_constant__ CUtensorMap map_q,
                   const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -253,9 +279,23 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
         if (t < np) { t = np - 1 - t; break; }
         t -= np;
     }
+    // last-token mode: a sequence without rows in this call gets zeros in its span_mass row
+    if (NS > 0 && blockIdx.x == 0 && blockIdx.y == 0 && a.probe_rows == HOOK_PROBE_ROWS_LAST) {
+        const int per = a.P * a.S;
+        for (int sq = warp; sq < a.num_seqs; sq += kThreads / 32) {
+            if (a.cu_q_lens[sq + 1] - a.cu_q_lens[sq] > 0) continue;
+            for (int i = lane; i < per; i += 32) a.mass[(int64_t)sq * per + i] = 0.f;
+        }
+    }
     if (s >= a.num_seqs) return;
     // once any CTA of this launch has given up on a wait, the rest of the grid does not start
-    if (a.status && *reinterpret_cast<volatile int32_t*>(a.status) == HOOK_ATTN_ERR_TIMEOUT) return;
+    {
+        const volatile LaunchAbort* ab = &g_launch_abort;
+        if (ab->launch_id == launch_id && global_timer_ns() - ab->when_ns < kAbortWindowNs) {
+            if (threadIdx.x == 0) report(a.status, HOOK_ATTN_ERR_TIMEOUT);
+            return;
+        }
+    }
     const int L = a.seq_lens[s];
     const int64_t grow_seq = a.cu_q_lens[s];
     const int row0[2] = {2 * t * kBM, (2 * t + 1) * kBM};
@@ -266,11 +306,21 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
         first_pos[x] = L - n + row0[x];
         ntiles[x] = rows[x] > 0 ? (first_pos[x] + rows[x] - 1) / kBN + 1 : 0;
     }
-    if (n > L || L > a.max_blocks * kPage) {
+    if (n > L || L > a.max_keys) {
         if (threadIdx.x == 0) report(a.status, n > L ? HOOK_ATTN_ERR_INVALID_ARG : HOOK_ATTN_ERR_BOUNDS);
         const int nrows = rows[0] + rows[1];
         for (int idx = threadIdx.x; idx < nrows * kHD; idx += kThreads)
             a.out[((grow_seq + row0[0] + idx / kHD) * a.Hq + h) * kHD + idx % kHD] = __float2bfloat16(0.f);
+        const int slot_bad = (NS > 0) ? hc.slot[h] : -1;
+        if (NS > 0 && slot_bad >= 0) {   // the probed rows of this tile pair: zeros as well
+            const bool last_only = (a.probe_rows == HOOK_PROBE_ROWS_LAST);
+            for (int idx = threadIdx.x; idx < nrows * a.S; idx += kThreads) {
+                const int r = row0[0] + idx / a.S, js = idx % a.S;
+                if (last_only && r != n - 1) continue;
+                const int64_t mrow = last_only ? (int64_t)s : grow_seq + r;
+                a.mass[(mrow * a.P + slot_bad) * a.S + js] = 0.f;
+            }
+        }
         return;
     }
     const int nmax = max(ntiles[0], ntiles[1]);
@@ -305,6 +355,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     bool ok = true;   // false once a bounded wait ran out
+    volatile int* abort_flag = &bars.abort_flag;
     const int32_t* bt = a.block_table + (int64_t)s * a.max_blocks;
     // producer: the loads of key tile j (K then V), one TMA box per (page, 64-wide half of the head)
     auto produce = [&](int j) {
@@ -321,7 +372,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
         for (int kv = 0; kv < 2; ++kv) {
             const uint32_t full = smem_u32(kv ? &bars.v_full[st] : &bars.k_full[st]);
             const uint32_t empty = smem_u32(kv ? &bars.v_empty[st] : &bars.k_empty[st]);
-            ok = __all_sync(0xffffffffu, mbar_wait(empty, ph ^ 1u));
+            ok = __all_sync(0xffffffffu, mbar_wait(empty, ph ^ 1u, abort_flag));
             if (!ok) break;
             if (lane == 0) mbar_expect_tx(full, (uint32_t)pages * 2u * (kPage * 128u));
             __syncwarp();
@@ -381,7 +432,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             // tensor cores: 0 * NaN would poison the accumulator.  Zero them in shared memory once the
             // last tile has landed, then tell the MMA thread.
             const int j = nmax - 1, st = j & 1;
-            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1));
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1, abort_flag));
             if (ok) {
                 const int r_first = L - j * kBN;
                 const uint32_t vb = sV + st * kTileBytes;
@@ -423,8 +474,8 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             // one thread runs the whole issue loop: no votes, no warp barriers on the pacemaker's path
 #pragma unroll
             for (int x = 0; x < 2; ++x)
-                if (ok && ntiles[x] > 0) ok = mbar_wait(smem_u32(&bars.q_full[x]), 0);
-            if (ok) ok = mbar_wait(smem_u32(&bars.k_full[0]), 0);
+                if (ok && ntiles[x] > 0) ok = mbar_wait(smem_u32(&bars.q_full[x]), 0, abort_flag);
+            if (ok) ok = mbar_wait(smem_u32(&bars.k_full[0]), 0, abort_flag);
             if (ok) {
                 tc_fence_after();
                 if (ntiles[0] > 0) issue_qk(0, 0);
@@ -432,13 +483,13 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             }
             for (int j = 0; j < nmax && ok; ++j) {
                 const int st = j & 1;
-                ok = mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1);
-                if (ok && j == nmax - 1 && (j + 1) * kBN > L) ok = mbar_wait(smem_u32(&bars.v_tail), 0);
-                if (ok && j + 1 < nmax) ok = mbar_wait(smem_u32(&bars.k_full[(j + 1) & 1]), ((j + 1) >> 1) & 1);
+                ok = mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1, abort_flag);
+                if (ok && j == nmax - 1 && (j + 1) * kBN > L) ok = mbar_wait(smem_u32(&bars.v_tail), 0, abort_flag);
+                if (ok && j + 1 < nmax) ok = mbar_wait(smem_u32(&bars.k_full[(j + 1) & 1]), ((j + 1) >> 1) & 1, abort_flag);
 #pragma unroll
                 for (int x = 0; x < 2; ++x) {
                     if (ok && j < ntiles[x]) {
-                        ok = mbar_wait(smem_u32(&bars.p_full[x]), j & 1);
+                        ok = mbar_wait(smem_u32(&bars.p_full[x]), j & 1, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
                         issue_pv(x, j);
@@ -468,7 +519,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             for (int js = 0; js < (NS > 0 ? NS : 1); ++js) sm[js] = 0.f;
 
             for (int j = 0; j < nt && ok; ++j) {
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), j & 1));
+                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), j & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 if (releases && (threadIdx.x & 127) == 0) {
@@ -588,7 +639,7 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
             }
 
             // ---- epilogue: normalise, steer, round once, store ----
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_full[x]), 0));
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_full[x]), 0, abort_flag));
             const float inv = 1.f / l;
             const bool live = row < rows[x];
             const uint32_t stage = sQ[x];
@@ -653,8 +704,11 @@ prefill_tc_kernel(const KernelArgs a, const HeadCfg hc, const __grid_constant__ 
 
     // ---- teardown ----
     if (!ok) {
-        if (lane == 0) report(a.status, HOOK_ATTN_ERR_TIMEOUT);
-        atomicExch(&bars.abort_flag, 1);
+        if (lane == 0) {
+            report(a.status, HOOK_ATTN_ERR_TIMEOUT);
+            g_launch_abort.launch_id = launch_id;
+            g_launch_abort.when_ns = global_timer_ns();
+        }
         const uint64_t t0 = global_timer_ns();           // let copies that are still in flight land
         while (global_timer_ns() - t0 < 1000000ull) __nanosleep(1000);
     }
@@ -693,22 +747,61 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-bool encode(CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
-            const cuuint32_t* box)
+// What a descriptor is made from; descriptors are cached under it.
+struct TmapKey {
+    const void* base;
+    uint32_t rank;
+    uint32_t box[4];
+    uint64_t dims[4];
+    uint64_t strides[3];   // bytes
+};
+
+struct TmapCache {
+    static constexpr size_t kEntries = 256;   // a model's layers times q/k/v; replaced round-robin beyond that
+    std::mutex mu;
+    std::vector<std::pair<TmapKey, CUtensorMap>> entries;
+    size_t next = 0;
+};
+
+// The descriptor of a bf16 tensor with 128B-swizzled boxes: from the cache when the same base pointer,
+// shape and strides were seen before (a serving loop re-issues the same layers), encoded otherwise.
+bool tensor_map(TmapCache* cache, CUtensorMap* map, const void* base, int rank, const cuuint64_t* dims,
+                const cuuint64_t* strides_bytes, const cuuint32_t* box)
 {
+    TmapKey key;
+    memset(&key, 0, sizeof key);
+    key.base = base;
+    key.rank = (uint32_t)rank;
+    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides_bytes[i];
+    if (cache) {
+        std::lock_guard<std::mutex> lock(cache->mu);
+        for (const auto& e : cache->entries)
+            if (memcmp(&e.first, &key, sizeof key) == 0) { *map = e.second; return true; }
+    }
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box, ones,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box, ones,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    if (cache) {
+        std::lock_guard<std::mutex> lock(cache->mu);
+        if (cache->entries.size() < TmapCache::kEntries) cache->entries.emplace_back(key, *map);
+        else { cache->entries[cache->next] = std::make_pair(key, *map); cache->next = (cache->next + 1) % TmapCache::kEntries; }
+    }
+    return true;
 }
+
+std::atomic<unsigned int> g_launch_counter{1};
 
 template <int NS>
 cudaError_t launch_t(const KernelArgs& a, const HeadCfg& hc, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                      int pairs, cudaStream_t st)
 {
-    prefill_tc_kernel<NS><<<dim3(a.Hq, pairs), kThreads, kSmemBytes, st>>>(a, hc, mq, mk, mv);
+    const unsigned int launch_id = g_launch_counter.fetch_add(1, std::memory_order_relaxed);
+    prefill_tc_kernel<NS><<<dim3(a.Hq, pairs), kThreads, kSmemBytes, st>>>(a, hc, launch_id, mq, mk, mv);
     return cudaGetLastError();
 }
 
@@ -719,6 +812,9 @@ cudaError_t configure_one()
 }
 
 }  // namespace
+
+void* tmap_cache_create() { return new TmapCache; }
+void tmap_cache_destroy(void* cache) { delete static_cast<TmapCache*>(cache); }
 
 // Self-test of the bounded waits: one CTA waits on an mbarrier that nothing ever arrives at.  The
 // wait must run out after `limit_ns`, the kernel must report HOOK_ATTN_ERR_TIMEOUT through the status
@@ -732,7 +828,7 @@ __global__ void wait_selftest_kernel(int32_t* status, uint64_t limit_ns, uint64_
     }
     __syncthreads();
     const uint64_t t0 = global_timer_ns();
-    const bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar), 0, limit_ns));
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar), 0, nullptr, limit_ns));
     if (threadIdx.x == 0) {
         if (!ok) report(status, HOOK_ATTN_ERR_TIMEOUT);
         if (waited_ns) *waited_ns = global_timer_ns() - t0;
@@ -761,24 +857,26 @@ bool prefill_tc_supported(const KernelArgs& a, int head_dim)
            a.bs < (1ll << 38) && a.ts < (1ll << 38) && a.hs < (1ll << 38);
 }
 
-cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, cudaStream_t st)
+cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, void* tmap_cache, int num_sms, cudaStream_t st)
 {
+    TmapCache* cache = static_cast<TmapCache*>(tmap_cache);
     CUtensorMap mq, mk, mv;
     {
         const cuuint64_t dims[3] = {(cuuint64_t)kHD, (cuuint64_t)a.Hq, (cuuint64_t)a.total_q};
         const cuuint64_t strides[2] = {(cuuint64_t)kHD * 2, (cuuint64_t)a.Hq * kHD * 2};
         const cuuint32_t box[3] = {64, 1, (cuuint32_t)kBM};
-        if (!encode(&mq, a.q, 3, dims, strides, box)) return cudaErrorInvalidValue;
+        if (!tensor_map(cache, &mq, a.q, 3, dims, strides, box)) return cudaErrorInvalidValue;
     }
     {
         const cuuint64_t dims[4] = {(cuuint64_t)kHD, (cuuint64_t)a.Hkv, (cuuint64_t)kPage, (cuuint64_t)a.num_blocks};
         const cuuint64_t strides[3] = {(cuuint64_t)a.hs * 2, (cuuint64_t)a.ts * 2, (cuuint64_t)a.bs * 2};
         const cuuint32_t box[4] = {64, 1, (cuuint32_t)kPage, 1};
-        if (!encode(&mk, a.k, 4, dims, strides, box)) return cudaErrorInvalidValue;
-        if (!encode(&mv, a.v, 4, dims, strides, box)) return cudaErrorInvalidValue;
+        if (!tensor_map(cache, &mk, a.k, 4, dims, strides, box)) return cudaErrorInvalidValue;
+        if (!tensor_map(cache, &mv, a.v, 4, dims, strides, box)) return cudaErrorInvalidValue;
     }
     // sum over sequences of ceil(n_s / 256) <= floor(total_q / 256) + num_seqs
     const int pairs = a.total_q / (2 * kBM) + a.num_seqs;
+    (void)num_sms;
     const int ns = !a.any_probe ? 0 : (a.S <= 2 ? 2 : (a.S <= 4 ? 4 : 8));
     switch (ns) {
         case 0: return launch_t<0>(a, hc, mq, mk, mv, pairs, st);

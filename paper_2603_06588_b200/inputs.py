@@ -20,7 +20,11 @@ Conventions (shared by every consumer):
 * ``alpha``       fp32 ``[Hq]``, ``steer_vec`` fp32 ``[Hq, D]`` -- per-head steering.
 
 All values are drawn in fp32 from a ``torch.Generator`` on the CPU and rounded to bf16
-once; those bf16 bits are what every consumer reads.
+once; those bf16 bits are what every consumer reads.  With ``device="cuda"`` the large
+tensors (queries, K/V pages, page permutation) are drawn by a seeded generator of that
+device instead -- the same recipe and distributions, other values -- which turns seconds
+of host-side drawing into milliseconds for the benchmark's largest workloads;
+:func:`to_host` gives the CPU copy of such a case for the oracle.
 """
 from __future__ import annotations
 
@@ -96,8 +100,8 @@ class HookAttnCase:
 # building blocks
 # ----------------------------------------------------------------------------------------
 
-def _gen(seed: int) -> torch.Generator:
-    g = torch.Generator(device="cpu")
+def _gen(seed: int, device="cpu") -> torch.Generator:
+    g = torch.Generator(device=device)
     g.manual_seed(int(seed))
     return g
 
@@ -108,10 +112,10 @@ def _randn_bf16(shape: Sequence[int], g: torch.Generator, std: float = 1.0,
     n = 1
     for s in shape:
         n *= int(s)
-    out = torch.empty(n, dtype=torch.bfloat16)
+    out = torch.empty(n, dtype=torch.bfloat16, device=g.device)
     for lo in range(0, n, chunk):
         hi = min(n, lo + chunk)
-        x = torch.randn(hi - lo, generator=g, dtype=torch.float32)
+        x = torch.randn(hi - lo, generator=g, dtype=torch.float32, device=g.device)
         if std != 1.0:
             x.mul_(std)
         out[lo:hi] = x.to(torch.bfloat16)
@@ -135,11 +139,12 @@ def paged_cache(seq_lens: Sequence[int], num_kv_heads: int, head_dim: int, g: to
     if max_blocks is not None:
         assert max_blocks >= mb
         mb = max_blocks
-    perm = torch.randperm(num_blocks, generator=g) if shuffle else torch.arange(num_blocks)
-    block_table = torch.full((len(seq_lens), mb), -1, dtype=torch.int32)
+    dev = g.device
+    perm = torch.randperm(num_blocks, generator=g, device=dev) if shuffle else torch.arange(num_blocks, device=dev)
+    block_table = torch.full((len(seq_lens), mb), -1, dtype=torch.int32, device=dev)
     fill = float("nan") if poison else 0.0
-    k_cache = torch.full((num_blocks, PAGE, num_kv_heads, head_dim), fill, dtype=torch.bfloat16)
-    v_cache = torch.full((num_blocks, PAGE, num_kv_heads, head_dim), fill, dtype=torch.bfloat16)
+    k_cache = torch.full((num_blocks, PAGE, num_kv_heads, head_dim), fill, dtype=torch.bfloat16, device=dev)
+    v_cache = torch.full((num_blocks, PAGE, num_kv_heads, head_dim), fill, dtype=torch.bfloat16, device=dev)
     cursor = 0
     for s, L in enumerate(seq_lens):
         np_s = pages[s]
@@ -152,7 +157,7 @@ def paged_cache(seq_lens: Sequence[int], num_kv_heads: int, head_dim: int, g: to
         v = _randn_bf16((L, num_kv_heads, head_dim), g, v_std)
         pad = np_s * PAGE - L
         if pad:
-            tail = torch.full((pad, num_kv_heads, head_dim), fill, dtype=torch.bfloat16)
+            tail = torch.full((pad, num_kv_heads, head_dim), fill, dtype=torch.bfloat16, device=dev)
             k = torch.cat([k, tail], 0)
             v = torch.cat([v, tail], 0)
         k_cache[phys] = k.view(np_s, PAGE, num_kv_heads, head_dim)
@@ -197,9 +202,13 @@ def make_case(name: str, *, is_decode: bool, seq_lens: Sequence[int], q_lens: Se
               steer: bool = False, probe_rows: int = PROBE_ROWS_ALL,
               q_std: float = 1.0, k_std: float = 1.0, v_std: float = 1.0,
               poison: bool = False, shuffle: bool = True, pool: float = 1.25,
-              max_blocks: Optional[int] = None, scale: Optional[float] = None) -> HookAttnCase:
-    """Generic seeded case builder used by the named configurations and by the tests."""
-    g = _gen(seed)
+              max_blocks: Optional[int] = None, scale: Optional[float] = None,
+              device: str = "cpu") -> HookAttnCase:
+    """Generic seeded case builder used by the named configurations and by the tests.  ``device``
+    other than ``"cpu"`` draws q, K/V and the page permutation with that device's generator (the small
+    host-side arrays stay on the CPU and come from a CPU generator of the same seed)."""
+    g = _gen(seed, device)
+    g_host = g if str(device) == "cpu" else _gen(seed)
     seq_lens = [int(x) for x in seq_lens]
     q_lens = [int(x) for x in q_lens]
     assert len(seq_lens) == len(q_lens)
@@ -209,10 +218,10 @@ def make_case(name: str, *, is_decode: bool, seq_lens: Sequence[int], q_lens: Se
     tq = sum(q_lens)
     q = _randn_bf16((tq, num_q_heads, head_dim), g, q_std)
     if spans is None and num_spans > 0:
-        spans = partition_spans(seq_lens, num_spans, g)
+        spans = partition_spans(seq_lens, num_spans, g_host)
     steer_vec = None
     if steer:
-        steer_vec = torch.randn((num_q_heads, head_dim), generator=g, dtype=torch.float32)
+        steer_vec = torch.randn((num_q_heads, head_dim), generator=g_host, dtype=torch.float32)
     if spans is not None:
         num_spans = int(spans.shape[1])
     return HookAttnCase(
@@ -245,7 +254,7 @@ def config1_tiny_prefill(poison: bool = False) -> HookAttnCase:
 
 
 def config2_decode(num_seqs: int = 64, lo: int = 512, hi: int = 4096, poison: bool = False,
-                   seed_offset: int = 0) -> HookAttnCase:
+                   seed_offset: int = 0, device: str = "cpu") -> HookAttnCase:
     seed = BASE_SEED + 2 + seed_offset
     g = _gen(seed ^ 0x5EED)
     Hq, Hkv, D = 32, 8, 128
@@ -261,7 +270,7 @@ def config2_decode(num_seqs: int = 64, lo: int = 512, hi: int = 4096, poison: bo
     return make_case("cfg2_decode", is_decode=True, seq_lens=L, q_lens=[1] * num_seqs,
                      num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, seed=seed, spans=spans,
                      head_mask=head_mask, alpha=alpha, steer=True,
-                     probe_rows=PROBE_ROWS_LAST, poison=poison)
+                     probe_rows=PROBE_ROWS_LAST, poison=poison, device=device)
 
 
 def config3_layer_masks(num_layers: int = 32, num_heads: int = 32, frac: float = 0.10) -> torch.Tensor:
@@ -275,7 +284,7 @@ def config3_layer_masks(num_layers: int = 32, num_heads: int = 32, frac: float =
 
 
 def config3_prefill(layer: int = 0, num_seqs: int = 8, tokens: int = 4096,
-                    poison: bool = False, force_probe: bool = False) -> HookAttnCase:
+                    poison: bool = False, force_probe: bool = False, device: str = "cpu") -> HookAttnCase:
     seed = BASE_SEED + 3 + 1000 * layer
     Hq, Hkv, D = 32, 8, 128
     mask = config3_layer_masks()[layer % 32].clone()
@@ -284,7 +293,7 @@ def config3_prefill(layer: int = 0, num_seqs: int = 8, tokens: int = 4096,
     return make_case(f"cfg3_prefill_l{layer}", is_decode=False, seq_lens=[tokens] * num_seqs,
                      q_lens=[tokens] * num_seqs, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
                      seed=seed, num_spans=3, head_mask=mask, alpha=None, steer=False,
-                     probe_rows=PROBE_ROWS_ALL, k_std=128.0 ** -0.5, poison=poison)
+                     probe_rows=PROBE_ROWS_ALL, k_std=128.0 ** -0.5, poison=poison, device=device)
 
 
 def _config4_common(g: torch.Generator):
@@ -297,7 +306,7 @@ def _config4_common(g: torch.Generator):
 
 
 def config4_decode(num_seqs: int = 256, lo: int = 1024, hi: int = 8192,
-                   poison: bool = False) -> HookAttnCase:
+                   poison: bool = False, device: str = "cpu") -> HookAttnCase:
     seed = BASE_SEED + 4
     g = _gen(seed ^ 0x5EED)
     head_mask, alpha = _config4_common(g)
@@ -305,18 +314,18 @@ def config4_decode(num_seqs: int = 256, lo: int = 1024, hi: int = 8192,
     return make_case("cfg4_mixed_decode", is_decode=True, seq_lens=L, q_lens=[1] * num_seqs,
                      num_q_heads=28, num_kv_heads=4, head_dim=128, seed=seed, num_spans=4,
                      head_mask=head_mask, alpha=alpha, steer=True,
-                     probe_rows=PROBE_ROWS_LAST, poison=poison)
+                     probe_rows=PROBE_ROWS_LAST, poison=poison, device=device)
 
 
 def config4_prefill(chunks: int = 2, n: int = 2048, ctx: int = 4096,
-                    poison: bool = False) -> HookAttnCase:
+                    poison: bool = False, device: str = "cpu") -> HookAttnCase:
     seed = BASE_SEED + 4 + 500
     g = _gen((BASE_SEED + 4) ^ 0x5EED)
     head_mask, alpha = _config4_common(g)
     return make_case("cfg4_mixed_prefill", is_decode=False, seq_lens=[ctx + n] * chunks,
                      q_lens=[n] * chunks, num_q_heads=28, num_kv_heads=4, head_dim=128,
                      seed=seed, num_spans=4, head_mask=head_mask, alpha=alpha, steer=True,
-                     probe_rows=PROBE_ROWS_ALL, poison=poison)
+                     probe_rows=PROBE_ROWS_ALL, poison=poison, device=device)
 
 
 def _config5_common(probed: int):
@@ -329,16 +338,16 @@ def _config5_common(probed: int):
 
 
 def config5_prefill(num_seqs: int = 4, tokens: int = 32768, probed: int = 64,
-                    poison: bool = False) -> HookAttnCase:
+                    poison: bool = False, device: str = "cpu") -> HookAttnCase:
     head_mask, alpha = _config5_common(probed)
     return make_case("cfg5_long_prefill", is_decode=False, seq_lens=[tokens] * num_seqs,
                      q_lens=[tokens] * num_seqs, num_q_heads=64, num_kv_heads=8, head_dim=128,
                      seed=BASE_SEED + 5, num_spans=8, head_mask=head_mask, alpha=alpha,
-                     steer=True, probe_rows=PROBE_ROWS_ALL, poison=poison)
+                     steer=True, probe_rows=PROBE_ROWS_ALL, poison=poison, device=device)
 
 
 def config5_decode(num_seqs: int = 4, tokens: int = 32768, steps: int = 128, step: int = 0,
-                   probed: int = 64, poison: bool = False) -> HookAttnCase:
+                   probed: int = 64, poison: bool = False, device: str = "cpu") -> HookAttnCase:
     """Decode step ``step`` of the long-context workload.  The cache is pre-filled to
     ``tokens + steps`` keys so that no append is part of a step; step ``t`` sees
     ``tokens + t + 1`` keys (its own row included)."""
@@ -347,8 +356,33 @@ def config5_decode(num_seqs: int = 4, tokens: int = 32768, steps: int = 128, ste
     case = make_case("cfg5_long_decode", is_decode=True, seq_lens=[cap] * num_seqs,
                      q_lens=[1] * num_seqs, num_q_heads=64, num_kv_heads=8, head_dim=128,
                      seed=BASE_SEED + 5 + 500, num_spans=8, head_mask=head_mask, alpha=alpha,
-                     steer=True, probe_rows=PROBE_ROWS_LAST, poison=poison)
+                     steer=True, probe_rows=PROBE_ROWS_LAST, poison=poison, device=device)
     return with_seq_lens(case, [tokens + step + 1] * num_seqs)
+
+
+def config5_session(num_seqs: int = 4, tokens: int = 32768, steps: int = 128, probed: int = 64,
+                    device: str = "cpu"):
+    """The long-context workload as one session on one cache: a full causal prefill of ``tokens`` keys per
+    sequence followed by ``steps`` decode steps.  The cache is pre-filled to ``tokens + steps`` keys so that
+    no append is part of a step.  Returns ``(prefill_case, [decode case of step 0 .. steps-1])``; all cases
+    share the K/V pages, the block table, the head mask and the steering."""
+    dec0 = config5_decode(num_seqs=num_seqs, tokens=tokens, steps=steps, step=0, probed=probed, device=device)
+    g_dev = _gen(BASE_SEED + 5, device)
+    g_host = _gen(BASE_SEED + 5 + 7)
+    q_pf = _randn_bf16((num_seqs * tokens, dec0.num_q_heads, dec0.head_dim), g_dev)
+    prefill = replace(dec0, name="cfg5_long_prefill", is_decode=False, q=q_pf,
+                      seq_lens=torch.tensor([tokens] * num_seqs, dtype=torch.int32),
+                      cu_q_lens=_cu([tokens] * num_seqs),
+                      spans=partition_spans([tokens] * num_seqs, dec0.num_spans, g_host),
+                      probe_rows=PROBE_ROWS_ALL)
+    decodes = [with_seq_lens(dec0, [tokens + t + 1] * num_seqs) for t in range(steps)]
+    return prefill, decodes
+
+
+def to_host(case: HookAttnCase) -> HookAttnCase:
+    """The same case with every tensor on the CPU (for consumers that read host memory)."""
+    moved = {f: getattr(case, f).cpu() for f in ("q", "k_cache", "v_cache", "block_table")}
+    return replace(case, **moved)
 
 
 def with_seq_lens(case: HookAttnCase, seq_lens: Sequence[int]) -> HookAttnCase:

@@ -79,6 +79,7 @@ def _params(**over):
     (dict(num_q_heads=32, num_kv_heads=2), binding.HOOK_ATTN_ERR_UNSUPPORTED),   # group 16
     (dict(num_spans=9), binding.HOOK_ATTN_ERR_UNSUPPORTED),
     (dict(num_seqs=-1), binding.HOOK_ATTN_ERR_INVALID_ARG),
+    (dict(max_seq_len=-1), binding.HOOK_ATTN_ERR_INVALID_ARG),
     (dict(probe_rows=7), binding.HOOK_ATTN_ERR_INVALID_ARG),
     (dict(q=None), binding.HOOK_ATTN_ERR_INVALID_ARG),
     (dict(out=None), binding.HOOK_ATTN_ERR_INVALID_ARG),
@@ -118,6 +119,9 @@ def test_decode_shape_and_workspace_checks(lib):
     p.workspace, p.workspace_bytes = 0x20000, need - 1
     assert lib.hook_attn_decode(None, ctypes.byref(p), None) == binding.HOOK_ATTN_ERR_WORKSPACE
     p.workspace_bytes = need
+    p.workspace = 0x20010                                    # the header asks for 256-byte alignment
+    assert lib.hook_attn_decode(None, ctypes.byref(p), None) == binding.HOOK_ATTN_ERR_WORKSPACE
+    p.workspace = 0x20000
     # everything valid except the handle: still refused, and nothing was launched
     assert lib.hook_attn_decode(None, ctypes.byref(p), None) == binding.HOOK_ATTN_ERR_INVALID_ARG
     # invalid shapes size to zero
@@ -131,6 +135,60 @@ def test_workspace_scales_with_the_bounds(lib):
     b = lib.hook_attn_workspace_bytes(ctypes.byref(_params(num_seqs=8, total_q=8)), 1)
     c = lib.hook_attn_workspace_bytes(ctypes.byref(_params(num_seqs=12, total_q=12)), 1)
     assert a > 0 and c - b == b - a > 0
+
+
+def test_length_bound_sizes_the_workspace_instead_of_the_table_width(lib):
+    """A block table padded to a model's maximum length must not inflate the plan: with the host's bound
+    on the sequence lengths the workspace is the one of the tight table."""
+    tight = lib.hook_attn_workspace_bytes(ctypes.byref(_params(num_seqs=64, total_q=64, max_blocks_per_seq=256)), 1)
+    padded = lib.hook_attn_workspace_bytes(ctypes.byref(_params(num_seqs=64, total_q=64, max_blocks_per_seq=8192)), 1)
+    hinted = lib.hook_attn_workspace_bytes(
+        ctypes.byref(_params(num_seqs=64, total_q=64, max_blocks_per_seq=8192, max_seq_len=4096)), 1)
+    assert padded > tight and hinted == tight
+    # a bound beyond what the table can address changes nothing
+    same = lib.hook_attn_workspace_bytes(
+        ctypes.byref(_params(num_seqs=64, total_q=64, max_blocks_per_seq=256, max_seq_len=1 << 20)), 1)
+    assert same == tight
+
+
+@pytest.mark.gpu
+def test_the_handles_device_must_be_current():
+    """Every entry point that launches refuses a handle whose device is not the current one.  The box has
+    one GPU, so the test edits the device ordinal the handle remembers (its first field) instead of
+    switching devices, and puts it back."""
+    from paper_2603_06588_b200 import inputs
+    eng = binding.HookAttn(0)
+    lib_ = binding.load_library()
+    case = inputs.config2_decode(num_seqs=2, lo=20, hi=60)
+    kw = binding.case_to_device(case)
+    plan = eng.plan(True, **kw)
+    plan.run()
+    torch.cuda.synchronize()
+    field = ctypes.cast(eng._h, ctypes.POINTER(ctypes.c_int))
+    assert field[0] == 0
+    field[0] = 1
+    try:
+        stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+        ref = ctypes.byref(plan.params)
+        assert lib_.hook_attn_decode(eng._h, ref, stream) == binding.HOOK_ATTN_ERR_INVALID_ARG
+        assert lib_.hook_attn_decode_static_scratch(eng._h, ref, stream) == binding.HOOK_ATTN_ERR_INVALID_ARG
+        pf = inputs.config3_prefill(layer=0, num_seqs=1, tokens=256, force_probe=True)
+        pkw = binding.case_to_device(pf)
+        pout = torch.empty_like(pkw["q"])
+        pmass = torch.zeros(pf.total_q, pf.num_probed, pf.num_spans, device="cuda")
+        pp, _keep = binding.make_params(out=pout, span_mass=pmass, **pkw)
+        assert lib_.hook_attn_prefill(eng._h, ctypes.byref(pp), stream) == binding.HOOK_ATTN_ERR_INVALID_ARG
+        m = torch.zeros(2, 2, 2, device="cuda")
+        assert lib_.hook_attn_score(eng._h, m.data_ptr(), 2, 2, 2, 1, m.data_ptr(), stream) == binding.HOOK_ATTN_ERR_INVALID_ARG
+        h = torch.zeros(4, 16, dtype=torch.bfloat16, device="cuda")
+        v = torch.zeros(16, device="cuda")
+        assert lib_.hook_steer_residual(eng._h, h.data_ptr(), v.data_ptr(), 1.0, 4, 16, 16, stream) == binding.HOOK_ATTN_ERR_INVALID_ARG
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        assert lib_.hook_attn_selftest_wait_limit(eng._h, st.data_ptr(), 1000, None, stream) == binding.HOOK_ATTN_ERR_INVALID_ARG
+    finally:
+        field[0] = 0
+    plan.run()                                                # the handle works again
+    torch.cuda.synchronize()
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="only meaningful without a GPU")

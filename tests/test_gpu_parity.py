@@ -395,6 +395,93 @@ def test_small_head_dim_128_calls_take_the_warp_mma_kernel(eng):
     check(eng, case)
 
 
+def test_padded_block_table_with_a_length_bound_gives_the_bits_of_the_tight_table(eng):
+    """Serving stacks pad block tables to the model's maximum length.  With the host's bound on the
+    lengths (`max_seq_len`) decode plans the same cut as for the tight table: same bits, and a workspace
+    of the same size.  Without the bound the padded table still gives correct results."""
+    case = inputs.config2_decode(poison=True)
+    kw = binding.case_to_device(case)
+    tight = eng.plan(True, **kw)
+    tight.run()
+    wide = torch.full((case.num_seqs, 8192), -1, dtype=torch.int32, device="cuda")
+    wide[:, :case.max_blocks_per_seq] = kw["block_table"]
+    kw_wide = dict(kw, block_table=wide)
+    hinted = eng.plan(True, max_seq_len=int(case.seq_lens.max()), **kw_wide)
+    hinted.run()
+    unhinted = eng.plan(True, **kw_wide)
+    unhinted.run()
+    torch.cuda.synchronize()
+    assert hinted.params.workspace_bytes <= eng.workspace_bytes(tight.params, True) < unhinted.params.workspace_bytes
+    assert torch.equal(hinted.out.view(torch.int16), tight.out.view(torch.int16)) and torch.equal(hinted.span_mass, tight.span_mass)
+    assert (unhinted.out.float() - tight.out.float()).abs().max().item() <= TOL_OUT
+    assert (unhinted.span_mass - tight.span_mass).abs().max().item() <= TOL_MASS
+    # a sequence longer than the bound is refused by the device check: status set, its row zeroed
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    short = eng.plan(True, max_seq_len=int(case.seq_lens.max()) - 1, status=status, **kw_wide)
+    short.run()
+    torch.cuda.synchronize()
+    longest = int(case.seq_lens.argmax())
+    assert int(status.item()) == binding.HOOK_ATTN_ERR_BOUNDS and torch.all(short.out[longest] == 0)
+
+
+def test_span_mass_rows_the_call_owns_are_always_written(eng):
+    """The caller may hand over uninitialised span_mass memory: every row the call owns is written --
+    zeros for a sequence without rows in last-token mode and for a sequence the device check refuses."""
+    case = inputs.make_case("owned", is_decode=False, seq_lens=[300, 64, 200, 150], q_lens=[300, 0, 130, 150],
+                            num_q_heads=4, num_kv_heads=2, head_dim=128, seed=21, num_spans=3,
+                            head_mask=torch.tensor([1, 0, 1, 1], dtype=torch.uint8),
+                            probe_rows=inputs.PROBE_ROWS_LAST, poison=True)
+    kw = binding.case_to_device(case)
+    mass = torch.full((4, 3, 3), float("nan"), device="cuda")
+    out = torch.full_like(kw["q"], float("nan"))
+    eng.hook_attn_prefill(out=out, span_mass=mass, **kw)
+    torch.cuda.synchronize()
+    assert torch.isfinite(mass).all() and torch.isfinite(out.float()).all() and torch.all(mass[1] == 0)
+    _, ref_mass = oracle.run(case, rows=oracle.last_rows(case))
+    assert np.abs(mass[[0, 2, 3]].cpu().numpy() - ref_mass).max() <= TOL_MASS
+    # sequence 2 claims more rows than keys: refused, its rows and its span_mass row are zeros
+    bad = inputs.with_seq_lens(case, [300, 64, 100, 150])
+    kwb = binding.case_to_device(bad)
+    for mode, rows in ((inputs.PROBE_ROWS_LAST, 4), (inputs.PROBE_ROWS_ALL, bad.total_q)):
+        mass = torch.full((rows, 3, 3), float("nan"), device="cuda")
+        out = torch.full_like(kwb["q"], float("nan"))
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        eng.hook_attn_prefill(out=out, span_mass=mass, status=status, **dict(kwb, probe_rows=mode))
+        torch.cuda.synchronize()
+        assert int(status.item()) == binding.HOOK_ATTN_ERR_INVALID_ARG
+        assert torch.isfinite(out.float()).all() and torch.all(out[300:430] == 0)
+        sel = mass[2] if mode == inputs.PROBE_ROWS_LAST else mass[300:430]
+        assert torch.all(sel == 0)
+        keep = [0, 3] if mode == inputs.PROBE_ROWS_LAST else list(range(300)) + list(range(430, bad.total_q))
+        assert torch.isfinite(mass[keep]).all()
+
+
+def test_prefill_of_more_tile_pairs_than_the_kernel_sorts(eng):
+    """More than 1024 (sequence, tile pair) entries: the persistent kernel walks them in sequence order
+    instead of sorting them.  Many short sequences, a few long ones, some without rows."""
+    g = inputs._gen(77)
+    lens = torch.randint(1, 200, (1100,), generator=g).tolist()
+    qls = [L if i % 7 else 0 for i, L in enumerate(lens)]
+    lens[500], qls[500] = 1500, 700
+    lens[1099], qls[1099] = 900, 900
+    case = inputs.make_case("many_pairs", is_decode=False, seq_lens=lens, q_lens=qls, num_q_heads=2, num_kv_heads=1,
+                            head_dim=128, seed=78, num_spans=2, head_mask=torch.tensor([1, 1], dtype=torch.uint8),
+                            alpha=torch.tensor([0.0, 0.75]), steer=True, poison=True)
+    assert case.total_q // 256 + case.num_seqs > 1024
+    check(eng, case, rows=inputs.sample_rows(case, extra_random=1))
+
+
+def test_prefill_skewed_batch_on_the_sorted_schedule(eng):
+    """Sequences of very different lengths and chunk offsets in one call: the sorted list mixes them, ties
+    in the tile count included; every row is checked."""
+    seq_lens = [1290, 256, 257, 700, 640, 128, 1024, 513]
+    q_lens = [300, 256, 257, 700, 130, 128, 512, 1]
+    case = inputs.make_case("pf_skew", is_decode=False, seq_lens=seq_lens, q_lens=q_lens, num_q_heads=4, num_kv_heads=2,
+                            head_dim=128, seed=33, num_spans=5, head_mask=torch.tensor([0, 1, 1, 0], dtype=torch.uint8),
+                            alpha=torch.tensor([0.3, 0.0, -0.4, 0.0]), steer=True, poison=True)
+    check(eng, case)
+
+
 @pytest.mark.parametrize("seed", range(24))
 def test_random_shapes_sweep(eng, seed):
     """Seeded random batches: ragged lengths, chunk offsets that are not tile-aligned, empty sequences,
