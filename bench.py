@@ -60,7 +60,7 @@ WORKLOADS = {
                              "seeded 10% of the 1024 (layer, head) pairs probed, 3 spans; one step = 32 layer calls",
     "cfg4_decode": "mixed batch, decode call: 256 seqs, ctx U[1024,8192], Hq28/Hkv4, D128, 14 probed heads, 4 spans, 8 steered heads",
     "cfg4_prefill": "mixed batch, prefill call: 2 chunks of 2048 tokens on 4096-token contexts, Hq28/Hkv4, D128",
-    "cfg4_mixed": "mixed chunked batch: the 256-sequence decode call and the 2-chunk prefill call of one step together",
+    "cfg4_mixed": "mixed chunked batch: the 256-sequence decode batch and the 2 prefill chunks of one step in one call",
     # profiling sizes and the companions of the attention path (only with --workload)
     "cfg3_prefill": "prefill: 8 seqs x 4096 tokens causal, Hq32/Hkv8, D128, layer-0 probes, 3 spans, one layer call per step",
     "cfg3_prefill_small": "prefill, profiling size: 2 seqs x 2048 tokens causal, Hq32/Hkv8, D128, layer-0 probes, 3 spans",
@@ -278,29 +278,36 @@ def build_layers(ctx, binding, layers=32):
 
 
 def build_mixed(ctx, binding):
+    """The mixed chunked batch as one call (hook_attn_mixed: one launch carries the decode batch and the prefill
+    chunks, a second one merges the decode partials).  The same two halves as two calls on two streams are
+    timed beside it (`two_stream_ms`)."""
     dec, pf = inputs.config4_decode(device=ctx.device), inputs.config4_prefill(device=ctx.device)
-    dh, dp = ctx.plans(dec, binding)
-    ph, pp = ctx.plans(pf, binding)
+    kw_dec, kw_pf = binding.case_to_device(dec, ctx.device), binding.case_to_device(pf, ctx.device)
+    hooks = ("spans", "head_mask", "alpha", "steer_vec")
+    fused = ctx.eng.mixed_plan(dict(kw_pf, status=ctx.status), dict(kw_dec, status=ctx.status))
+    plain = ctx.eng.mixed_plan({k: v for k, v in kw_pf.items() if k not in hooks},
+                               {k: v for k, v in kw_dec.items() if k not in hooks})
+    dh, _ = ctx.plans(dec, binding)
+    ph, _ = ctx.plans(pf, binding)
     side = torch.cuda.Stream(device=ctx.device)
     fork, join = torch.cuda.Event(), torch.cuda.Event()
 
-    def both(d, p):
-        def step():
-            main_s = torch.cuda.current_stream()
-            fork.record(main_s)
-            side.wait_event(fork)
-            with torch.cuda.stream(side):
-                p.run()
-                join.record(side)
-            d.run()
-            main_s.wait_event(join)
-        return step
+    def two_streams():
+        main_s = torch.cuda.current_stream()
+        fork.record(main_s)
+        side.wait_event(fork)
+        with torch.cuda.stream(side):
+            ph.run()
+            join.record(side)
+        dh.run()
+        main_s.wait_event(join)
     bytes_dec, _ = algorithmic_work(dec)
     _, flops_pf = algorithmic_work(pf)
-    return {"hooked": both(dh, ph), "plain": both(dp, pp), "tokens": dec.total_q + pf.total_q, "bound": "hbm", "work": bytes_dec,
-            "kernel": "decode_splitk_kernel + decode_merge_kernel on one stream, prefill_tc_kernel on a second; the bytes are "
-                      "the decode call's, over the time of the whole step",
-            "launches": 3, "keep": (dh, dp, ph, pp), "extra": {"prefill_flops_per_step": flops_pf}}
+    return {"hooked": fused.run, "plain": plain.run, "alt": two_streams, "tokens": dec.total_q + pf.total_q, "bound": "hbm",
+            "work": bytes_dec,
+            "kernel": "mixed_kernel (decode CTAs and prefill CTAs in one launch) + decode_merge_kernel; the bytes are the decode "
+                      "half's, over the time of the whole step",
+            "launches": 2, "keep": (fused, plain, dh, ph), "extra": {"prefill_flops_per_step": flops_pf}}
 
 
 class Session:
@@ -395,6 +402,9 @@ def measure_entry(ctx, name, w, warmup, sampler_windows, steps_per_block=0, bloc
         extra = dict(w.get("extra", {}))
         if "prefill_flops_per_step" in extra:
             extra["prefill_tflops_over_the_step"] = extra.pop("prefill_flops_per_step") / per_step / 1e12
+        if "alt" in w:
+            (ta,), _, _ = time_blocks([w["alt"]], warmup=warmup, blocks=blocks)
+            extra["two_stream_ms"] = statistics.median(ta) * 1e3
     # median of the ratios of neighbouring (hooked, plain) blocks: clock drift moves both members of a pair alike
     overhead = statistics.median(h / p for h, p in zip(th, tp)) - 1.0
     entry = {"workload": WORKLOADS[name], "tokens_per_step": w["tokens"], "tokens_per_s": w["tokens"] / per_step}

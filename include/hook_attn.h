@@ -128,8 +128,8 @@ int hook_attn_destroy(hook_attn_handle* handle);
 
 /* Bytes of scratch the call described by `p` needs (only the shape fields and max_seq_len are read;
  * pass the same max_seq_len to the call).
- * is_decode != 0 sizes hook_attn_decode, 0 sizes hook_attn_prefill.  Returns 0 when the call needs
- * no scratch or when the shapes are invalid. */
+ * is_decode = 1 sizes hook_attn_decode, 2 the decode half of hook_attn_mixed, 0 hook_attn_prefill.
+ * Returns 0 when the call needs no scratch or when the shapes are invalid. */
 size_t hook_attn_workspace_bytes(const hook_attn_params* p, int is_decode);
 
 /* Prefill / chunked prefill: n_s >= 0 rows per sequence given by cu_q_lens, n_s <= L_s.
@@ -145,6 +145,19 @@ int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void*
  * unit are merged in a fixed order, so results are bit-identical from run to run.  span_mass has one
  * row per sequence. */
 int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream);
+
+/* One step of a serving loop that holds both a decode batch and prefill chunks (chunked prefill, the
+ * usual shape of a served step): the work of hook_attn_decode(decode) and hook_attn_prefill(prefill), same
+ * arguments, outputs, results and error behaviour, issued together.  (Section 2: the hooks act inside the
+ * engine's forward pass, whatever mix of requests a step carries; Section 2.1: the worker runs them per
+ * execute_model call.)  When both halves have head_dim 128, the prefill half has at least 128 rows and the
+ * decode half at most 512 sequences, one launch carries both -- a part of the SMs streams the decode batch
+ * at HBM speed while the rest runs the prefill tiles on the tensor cores -- followed by the merge of the
+ * decode partials; otherwise the two calls are issued one after the other.  `decode->workspace` must hold
+ * hook_attn_workspace_bytes(decode, 2) bytes.  Either half may be empty (num_seqs = 0).  The two halves must
+ * not write overlapping outputs. */
+int hook_attn_mixed(hook_attn_handle* handle, const hook_attn_params* prefill, const hook_attn_params* decode,
+                    void* cuda_stream);
 
 /* Decode for callers that can neither allocate device memory nor hand over scratch.
  * (The paper has no counterpart; this is a convenience of the library.)

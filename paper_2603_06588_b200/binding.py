@@ -26,7 +26,7 @@ HOOK_PROBE_ROWS_ALL = 0
 HOOK_PROBE_ROWS_LAST = 1
 
 EXPORTS = ("hook_attn_create", "hook_attn_destroy", "hook_attn_workspace_bytes",
-           "hook_attn_prefill", "hook_attn_decode", "hook_attn_decode_static_scratch",
+           "hook_attn_prefill", "hook_attn_decode", "hook_attn_mixed", "hook_attn_decode_static_scratch",
            "hook_attn_score", "hook_steer_residual", "hook_capture_qk", "hook_attn_selftest_wait_limit",
            "hook_attn_strerror")
 HOOK_SCORE_MEAN = 0
@@ -83,6 +83,9 @@ def load_library() -> ctypes.CDLL:
             fn = getattr(lib, name)
             fn.restype = ctypes.c_int
             fn.argtypes = [ctypes.c_void_p, ctypes.POINTER(HookAttnParams), ctypes.c_void_p]
+        lib.hook_attn_mixed.restype = ctypes.c_int
+        lib.hook_attn_mixed.argtypes = [ctypes.c_void_p, ctypes.POINTER(HookAttnParams), ctypes.POINTER(HookAttnParams),
+                                        ctypes.c_void_p]
         lib.hook_attn_score.restype = ctypes.c_int
         lib.hook_attn_score.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                         ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
@@ -180,8 +183,9 @@ class HookAttn:
             pass
 
     # -- raw calls -----------------------------------------------------------------------
-    def workspace_bytes(self, params: HookAttnParams, is_decode: bool) -> int:
-        return int(self._lib.hook_attn_workspace_bytes(ctypes.byref(params), int(bool(is_decode))))
+    def workspace_bytes(self, params: HookAttnParams, is_decode) -> int:
+        """``is_decode``: False / True, or 2 for the decode half of a mixed step."""
+        return int(self._lib.hook_attn_workspace_bytes(ctypes.byref(params), int(is_decode)))
 
     def call(self, params: HookAttnParams, is_decode: bool, stream: Optional[int] = None) -> int:
         """Issue the call described by ``params``; returns the library's return code."""
@@ -268,7 +272,7 @@ class HookAttn:
     def plan(self, is_decode: bool, *, q, k_cache, v_cache, block_table, seq_lens, cu_q_lens=None,
              spans=None, head_mask=None, alpha=None, steer_vec=None, scale=0.0,
              probe_rows=HOOK_PROBE_ROWS_ALL, out=None, span_mass=None, status=None,
-             max_seq_len: int = 0) -> "HookAttnPlan":
+             max_seq_len: int = 0, mixed_half: bool = False) -> "HookAttnPlan":
         """Marshal the arguments once (allocating `out`, `span_mass` and scratch when they are not
         given); the returned plan re-issues the same call with one C call per step."""
         total_q, hq, d = q.shape
@@ -284,7 +288,7 @@ class HookAttn:
                               head_mask=head_mask, alpha=alpha, steer_vec=steer_vec, scale=scale,
                               probe_rows=probe_rows, out=out, span_mass=span_mass, status=status,
                               max_seq_len=max_seq_len)
-        nbytes = self.workspace_bytes(p, is_decode)
+        nbytes = self.workspace_bytes(p, 2 if (is_decode and mixed_half) else is_decode)
         ws = None
         if nbytes:
             ws = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
@@ -292,6 +296,16 @@ class HookAttn:
             p.workspace_bytes = nbytes
         keep += [q, k_cache, v_cache, block_table, seq_lens, cu_q_lens, spans, steer_vec, status, ws]
         return HookAttnPlan(self, is_decode, p, out, span_mass, keep)
+
+    def mixed_plan(self, prefill_kw: dict, decode_kw: dict) -> "HookAttnMixedPlan":
+        """A step with a decode batch and prefill chunks (``hook_attn_mixed``): marshals both halves once."""
+        return HookAttnMixedPlan(self, self.plan(False, **prefill_kw), self.plan(True, mixed_half=True, **decode_kw))
+
+    def hook_attn_mixed(self, prefill_kw: dict, decode_kw: dict):
+        """Returns ``((out, span_mass) of the prefill half, (out, span_mass) of the decode half)``."""
+        pl = self.mixed_plan(prefill_kw, decode_kw)
+        pl.run()
+        return (pl.prefill.out, pl.prefill.span_mass), (pl.decode.out, pl.decode.span_mass)
 
     def hook_attn_prefill(self, **kw):
         """Prefill / chunked prefill.  Returns ``(out, span_mass)``."""
@@ -321,6 +335,20 @@ class HookAttnPlan:
         rc = int(self._fn(self.eng._h, self._ref, ctypes.c_void_p(stream)))
         if rc != HOOK_ATTN_OK:
             raise HookAttnError(rc, "hook_attn_decode" if self.is_decode else "hook_attn_prefill")
+
+
+class HookAttnMixedPlan:
+    """The two marshalled halves of a mixed step; ``run()`` issues them with one ``hook_attn_mixed`` call."""
+
+    def __init__(self, eng: HookAttn, prefill: HookAttnPlan, decode: HookAttnPlan):
+        self.eng, self.prefill, self.decode = eng, prefill, decode
+
+    def run(self, stream: Optional[int] = None) -> None:
+        if stream is None:
+            stream = torch.cuda.current_stream(self.eng.device).cuda_stream
+        rc = int(self.eng._lib.hook_attn_mixed(self.eng._h, self.prefill._ref, self.decode._ref, ctypes.c_void_p(stream)))
+        if rc != HOOK_ATTN_OK:
+            raise HookAttnError(rc, "hook_attn_mixed")
 
 
 def case_to_device(case, device="cuda") -> dict:

@@ -23,6 +23,12 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, void* tmap
 void* tmap_cache_create();
 void tmap_cache_destroy(void* cache);
 cudaError_t launch_wait_selftest(int32_t* status, uint64_t limit_ns, uint64_t* waited_ns, cudaStream_t st);
+// mixed.cu
+cudaError_t configure_mixed();
+bool mixed_supported(const KernelArgs& apf, int head_dim_pf, const KernelArgs& adec, int head_dim_dec);
+size_t mixed_decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim);
+cudaError_t launch_mixed(const KernelArgs& apf, const HeadCfg& hpf, const KernelArgs& adec, const HeadCfg& hdec, void* tmap_cache,
+                         int num_sms, int forced_dec_ctas, cudaStream_t st);
 // extras.cu
 cudaError_t launch_score(const float* mass, float* scores, int rows, int P, int S, int mode, cudaStream_t st);
 cudaError_t launch_steer_residual(__nv_bfloat16* hidden, const float* vec, float alpha, int64_t tokens, int hidden_size,
@@ -39,6 +45,7 @@ struct hook_attn_handle {
     int cc_major, cc_minor;
     bool prefer_tc;   // head_dim-128 prefill goes to the tcgen05 kernel (HOOK_ATTN_PREFILL_KERNEL=mma turns it off)
     void* tmap_cache; // TMA descriptors of the prefill kernel, keyed by base pointer, shape and strides
+    int mixed_dec_ctas; // HOOK_ATTN_MIXED_DECODE_CTAS: CTAs in the decode role of the one-launch mixed step (0 = from the shapes)
 };
 
 namespace {
@@ -155,6 +162,7 @@ int hook_attn_create(hook_attn_handle** handle, int device)
     cudaError_t e = configure_decode();
     if (e == cudaSuccess) e = configure_prefill_mma();
     if (e == cudaSuccess) e = configure_prefill_tc();
+    if (e == cudaSuccess) e = configure_mixed();
     cudaSetDevice(prev);
     if (e != cudaSuccess) return HOOK_ATTN_ERR_CUDA;
     hook_attn_handle* h = new hook_attn_handle;
@@ -165,6 +173,8 @@ int hook_attn_create(hook_attn_handle** handle, int device)
     const char* pk = getenv("HOOK_ATTN_PREFILL_KERNEL");
     h->prefer_tc = !(pk && strcmp(pk, "mma") == 0);
     h->tmap_cache = tmap_cache_create();
+    const char* md = getenv("HOOK_ATTN_MIXED_DECODE_CTAS");
+    h->mixed_dec_ctas = md ? atoi(md) : 0;
     *handle = h;
     return HOOK_ATTN_OK;
 }
@@ -181,7 +191,12 @@ size_t hook_attn_workspace_bytes(const hook_attn_params* p, int is_decode)
     if (validate_common(p, is_decode != 0) != HOOK_ATTN_OK) return 0;
     if (!is_decode) return 0;
     const int G = p->num_q_heads / p->num_kv_heads;
-    return decode_workspace_bytes(p->num_seqs, p->num_kv_heads, G, p->head_dim, max_keys_of(p));
+    const size_t alone = decode_workspace_bytes(p->num_seqs, p->num_kv_heads, G, p->head_dim, max_keys_of(p));
+    if (is_decode != 2) return alone;
+    // the decode half of hook_attn_mixed: the one-launch path cuts by page shares whatever the unit count,
+    // the fallback is the stand-alone call
+    const size_t shared = mixed_decode_workspace_bytes(p->num_seqs, p->num_kv_heads, G, p->head_dim);
+    return alone > shared ? alone : shared;
 }
 
 int hook_attn_prefill(hook_attn_handle* handle, const hook_attn_params* p, void* cuda_stream)
@@ -216,6 +231,32 @@ int hook_attn_decode(hook_attn_handle* handle, const hook_attn_params* p, void* 
     if ((rc = check_handle(handle)) != HOOK_ATTN_OK) return rc;
     cudaError_t e = launch_decode(a, hc, p->head_dim, handle->num_sms, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
+}
+
+int hook_attn_mixed(hook_attn_handle* handle, const hook_attn_params* prefill, const hook_attn_params* decode, void* cuda_stream)
+{
+    KernelArgs apf, adec;
+    HeadCfg hpf, hdec;
+    int rc = prepare(prefill, false, apf, hpf);
+    if (rc != HOOK_ATTN_OK) return rc;
+    if ((rc = prepare(decode, true, adec, hdec)) != HOOK_ATTN_OK) return rc;
+    const bool has_pf = prefill->num_seqs > 0 && prefill->total_q > 0, has_dec = decode->num_seqs > 0;
+    if (has_dec && decode->max_blocks_per_seq == 0) return HOOK_ATTN_ERR_INVALID_ARG;
+    if (has_dec) {
+        const size_t need = hook_attn_workspace_bytes(decode, 2);
+        if (!decode->workspace || decode->workspace_bytes < need) return HOOK_ATTN_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(decode->workspace) & 255u) return HOOK_ATTN_ERR_WORKSPACE;
+    }
+    if ((rc = check_handle(handle)) != HOOK_ATTN_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (has_pf && has_dec && handle->prefer_tc && mixed_supported(apf, prefill->head_dim, adec, decode->head_dim)) {
+        cudaError_t e = launch_mixed(apf, hpf, adec, hdec, handle->tmap_cache, handle->num_sms, handle->mixed_dec_ctas, st);
+        return e == cudaSuccess ? HOOK_ATTN_OK : HOOK_ATTN_ERR_CUDA;
+    }
+    // shapes the one-launch kernel does not take (or an empty half): the two calls, one after the other
+    if (has_dec && (rc = hook_attn_decode(handle, decode, cuda_stream)) != HOOK_ATTN_OK) return rc;
+    if (has_pf && (rc = hook_attn_prefill(handle, prefill, cuda_stream)) != HOOK_ATTN_OK) return rc;
+    return HOOK_ATTN_OK;
 }
 
 // ---- decode without any caller-provided or allocated scratch --------------------------------

@@ -55,6 +55,74 @@ def test_steer_oracle_and_capture_oracle_by_brute_force():
     assert np.array_equal(q_out[2, 0], case.q[2, heads[0]].view(torch.int16).numpy())
 
 
+def test_the_two_readings_of_sum_normalize_differ():
+    """The paper names the reduction ("sum_normalize") and describes it in words only: attention on the
+    instruction against attention on instruction plus data, over the important heads.  Two formulas fit
+    those words.  (A, the library's) normalise every head's span masses by that head's total, then average
+    the heads: each head votes with equal weight.  (B) sum the masses over the heads first, then normalise
+    once: heads that put more mass on the configured spans weigh more.  They agree when all heads carry the
+    same total and differ otherwise; this test keeps the difference visible."""
+    m = np.array([[[0.10, 0.10], [0.60, 0.20]]])           # head 0: total 0.2, split 1:1; head 1: total 0.8, split 3:1
+    a = extras.scores(m, extras.SCORE_SUM_NORMALIZE)[0]
+    b = m[0].sum(axis=0) / m[0].sum()
+    assert np.allclose(a, [(0.5 + 0.75) / 2, (0.5 + 0.25) / 2])      # 0.625 / 0.375
+    assert np.allclose(b, [0.7, 0.3])
+    assert abs(a[0] - b[0]) > 0.05
+    same_totals = np.array([[[0.2, 0.2], [0.3, 0.1]]])                # both heads total 0.4: the readings coincide
+    assert np.allclose(extras.scores(same_totals, extras.SCORE_SUM_NORMALIZE)[0], same_totals[0].sum(0) / same_totals[0].sum())
+
+
+def _capture_by_loops(case):
+    """The capture payload written out with explicit loops over (sequence, key, probed head) on K gathered
+    contiguously by tests/_brute.py -- nothing shared with oracle/extras.py."""
+    from tests import _brute
+    hq, hkv, d = case.num_q_heads, case.num_kv_heads, case.head_dim
+    heads = [h for h in range(hq) if int(case.head_mask[h])]
+    cu_q = case.cu_q_lens.tolist()
+    lens = case.seq_lens.tolist()
+    last_only = case.is_decode or case.probe_rows == inputs.PROBE_ROWS_LAST
+    q = case.q.float().numpy()
+    k_rows, q_rows = [], []
+    for s in range(case.num_seqs):
+        k, _ = _brute.gather_contiguous(case, s)                       # [L, Hkv, D]
+        for t in range(lens[s]):
+            k_rows.append([[float(k[t, h // (hq // hkv), e]) for e in range(d)] for h in heads])
+        n = cu_q[s + 1] - cu_q[s]
+        if last_only:
+            q_rows.append([[float(q[cu_q[s + 1] - 1, h, e]) if n > 0 else 0.0 for e in range(d)] for h in heads])
+        else:
+            for i in range(n):
+                q_rows.append([[float(q[cu_q[s] + i, h, e]) for e in range(d)] for h in heads])
+    cu_k = [0]
+    for L in lens:
+        cu_k.append(cu_k[-1] + L)
+    return np.array(q_rows, dtype=np.float64).reshape(-1, len(heads), d), np.array(k_rows, dtype=np.float64).reshape(-1, len(heads), d), cu_k
+
+
+@pytest.mark.parametrize("mode", ["decode", "all_tokens", "last_token"])
+def test_capture_oracle_every_element_in_all_three_modes(mode):
+    """Tiny case, every element: a sequence without rows in the call, probed heads that skip a KV head and
+    share another (heads 0, 1 -> KV 0; 5 -> KV 2; 7 -> KV 3), sequence lengths that end inside a page."""
+    mask = torch.tensor([1, 1, 0, 0, 0, 1, 0, 1], dtype=torch.uint8)
+    if mode == "decode":
+        case = inputs.make_case("cap_pin_d", is_decode=True, seq_lens=[5, 33, 16], q_lens=[1, 1, 1], num_q_heads=8,
+                                num_kv_heads=4, head_dim=8, seed=41, head_mask=mask, poison=True)
+    else:
+        case = inputs.make_case("cap_pin_p", is_decode=False, seq_lens=[5, 33, 16, 20], q_lens=[5, 0, 3, 20], num_q_heads=8,
+                                num_kv_heads=4, head_dim=8, seed=42, head_mask=mask, poison=True,
+                                probe_rows=inputs.PROBE_ROWS_LAST if mode == "last_token" else inputs.PROBE_ROWS_ALL)
+    q_out, k_out, cu = extras.capture_qk(case)
+    want_q, want_k, want_cu = _capture_by_loops(case)
+    as_f = lambda bits: torch.from_numpy(np.ascontiguousarray(bits)).view(torch.bfloat16).float().numpy().astype(np.float64)
+    assert cu.tolist() == want_cu
+    assert q_out.shape == want_q.shape and k_out.shape == want_k.shape
+    assert np.array_equal(as_f(k_out), want_k)
+    assert np.array_equal(as_f(q_out), want_q)
+    if mode == "last_token":
+        assert not q_out[1].any()                                      # the sequence without rows: zeros
+        assert np.array_equal(as_f(q_out)[2, 3], case.q[7, 7].float().numpy())   # sequence 2's last row is global row 7
+
+
 def test_extras_reject_bad_arguments_without_a_gpu():
     lib = binding.load_library()
     assert lib.hook_attn_score(None, 0x1000, 4, 0, 2, 1, 0x1000, None) == binding.HOOK_ATTN_ERR_INVALID_ARG
