@@ -11,7 +11,7 @@
 //   warp  8    producer: resolves pages through the block table and issues one TMA box load per
 //              (page, 64-wide half of the head) into 128B-swizzled K and V stages; it also zeroes the
 //              value rows past the end of the sequence in the last tile;
-//   warp  9    owns tensor memory; one elected thread of it issues the MMAs: S = Q K^T (both operands
+//   warp  9    owns tensor memory and walks the issue loop as a whole; one elected lane of it issues the MMAs: S = Q K^T (both operands
 //              K-major in shared memory) and O += P V (P from tensor memory, V as the MN-major B
 //              operand), ordered PV(A,j) QK(A,j+1) PV(B,j) QK(B,j+1) so that one tile's softmax
 //              overlaps the other tile's tensor work.  That thread is the pacemaker of the CTA, so
@@ -466,28 +466,37 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
             for (int ks = 0; ks < kBN / 16; ++ks)
                 tc_mma_ts(tO[x], tS[x] + ks * 8, desc_advance(dv, (ks * 16 * 128) >> 4), idesc_pv, (ks > 0) || (j > 0));
         };
-        if (lane == 0) {
-            // one thread runs the whole issue loop: no votes, no warp barriers on the pacemaker's path
+        // The whole warp walks the issue loop in step -- every lane looks at the barriers, so loop counters,
+        // descriptors and branch conditions stay warp-uniform -- and one elected lane issues the MMAs and
+        // commits.  (A loop run by a single thread inside a divergent branch costs that thread several
+        // times the instructions per MMA; the tensor pipe's queue is shallow, so every cycle the issuing
+        // thread spends on anything else is a cycle the pipe idles.)  No votes: a lane whose wait runs out
+        // raises the abort flag, which ends the other lanes' waits as well.
+        uint32_t elected;
+        asm volatile("{\n\t.reg .pred pe;\n\telect.sync _|pe, 0xffffffff;\n\tselp.u32 %0, 1, 0, pe;\n\t}" : "=r"(elected));
 #pragma unroll
-            for (int x = 0; x < 2; ++x)
-                if (ok && ntiles[x] > 0) ok = mbar_wait(smem_u32(&bars.q_full[x]), 0, abort_flag);
-            if (ok) ok = mbar_wait(smem_u32(&bars.k_full[0]), 0, abort_flag);
-            if (ok) {
-                tc_fence_after();
+        for (int x = 0; x < 2; ++x)
+            if (ok && ntiles[x] > 0) ok = mbar_wait(smem_u32(&bars.q_full[x]), 0, abort_flag);
+        if (ok) ok = mbar_wait(smem_u32(&bars.k_full[0]), 0, abort_flag);
+        if (ok) {
+            tc_fence_after();
+            if (elected) {
                 if (ntiles[0] > 0) issue_qk(0, 0);
                 if (ntiles[1] > 0) issue_qk(1, 0);
             }
-            for (int j = 0; j < nmax && ok; ++j) {
-                const int st = j & 1;
-                ok = mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1, abort_flag);
-                if (ok && j == nmax - 1 && (j + 1) * kBN > L) ok = mbar_wait(smem_u32(&bars.v_tail), 0, abort_flag);
-                if (ok && j + 1 < nmax) ok = mbar_wait(smem_u32(&bars.k_full[(j + 1) & 1]), ((j + 1) >> 1) & 1, abort_flag);
+        }
+        for (int j = 0; j < nmax && ok; ++j) {
+            const int st = j & 1;
+            ok = mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1, abort_flag);
+            if (ok && j == nmax - 1 && (j + 1) * kBN > L) ok = mbar_wait(smem_u32(&bars.v_tail), 0, abort_flag);
+            if (ok && j + 1 < nmax) ok = mbar_wait(smem_u32(&bars.k_full[(j + 1) & 1]), ((j + 1) >> 1) & 1, abort_flag);
 #pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    if (ok && j < ntiles[x]) {
-                        ok = mbar_wait(smem_u32(&bars.p_full[x]), j & 1, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
+            for (int x = 0; x < 2; ++x) {
+                if (ok && j < ntiles[x]) {
+                    ok = mbar_wait(smem_u32(&bars.p_full[x]), j & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (elected) {
                         issue_pv(x, j);
                         if (j + 1 < ntiles[x]) issue_qk(x, j + 1);
                         else tc_commit(smem_u32(&bars.o_full[x]));
