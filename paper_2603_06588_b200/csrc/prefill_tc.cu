@@ -149,9 +149,7 @@ cudaError_t configure_prefill_tc()
 {
     cudaError_t e;
     if ((e = configure_one<0>()) != cudaSuccess) return e;
-    if ((e = configure_one<2>()) != cudaSuccess) return e;
-    if ((e = configure_one<4>()) != cudaSuccess) return e;
-    return configure_one<8>();
+    return configure_one<kMaxSpans>();
 }
 
 // True when the tensor-core kernel can serve the call (head_dim 128, tensor maps encodable).
@@ -188,13 +186,8 @@ cudaError_t launch_prefill_tc(const KernelArgs& a, const HeadCfg& hc, void* tmap
     CUtensorMap mq, mk, mv;
     if (!prefill_tc_maps(a, tmap_cache, &mq, &mk, &mv)) return cudaErrorInvalidValue;
     const int pairs = prefill_tc_pairs(a);
-    const int ns = !a.any_probe ? 0 : (a.S <= 2 ? 2 : (a.S <= 4 ? 4 : 8));
-    switch (ns) {
-        case 0: return launch_t<0>(a, hc, mq, mk, mv, pairs, st);
-        case 2: return launch_t<2>(a, hc, mq, mk, mv, pairs, st);
-        case 4: return launch_t<4>(a, hc, mq, mk, mv, pairs, st);
-        default: return launch_t<8>(a, hc, mq, mk, mv, pairs, st);
-    }
+    // two instantiations: without a probe, and with one (any number of spans: the span sums live in shared memory)
+    return a.any_probe ? launch_t<kMaxSpans>(a, hc, mq, mk, mv, pairs, st) : launch_t<0>(a, hc, mq, mk, mv, pairs, st);
 }
 
 }  // namespace hook_attn

@@ -240,6 +240,11 @@ struct LaunchAbort {
 static __device__ LaunchAbort g_launch_abort;
 constexpr unsigned long long kAbortWindowNs = 5000000000ull;
 
+template <bool B>
+struct ProbedTag {
+    static constexpr bool value = B;
+};
+
 struct Barriers {
     uint64_t q_full[2];
     uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
@@ -263,6 +268,8 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
     __shared__ Barriers bars;
     __shared__ int sh_span[2 * kMaxSpans];
     __shared__ uint16_t sh_tile_mask[kMaskTiles];   // per key tile: bits 0-7 spans covering it, bits 8-15 spans straddling it
+    __shared__ __align__(16) float sh_steer[kHD];    // alpha[h] * steer_vec[h][:] of a steered head
+    __shared__ float sh_sm[NS > 0 ? 2 : 1][NS > 0 ? kMaxSpans : 1][NS > 0 ? kBM : 1];   // span sums of tile x, span j, row r
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kvh = h / a.G;
@@ -393,6 +400,7 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
         }
         if (nmax > 0) produce(0);
     }
+    if (hc.alpha[h] != 0.f && (int)threadIdx.x < kHD) sh_steer[threadIdx.x] = hc.alpha[h] * a.steer[(int64_t)h * kHD + threadIdx.x];
     if (NS > 0 && (int)threadIdx.x < 2 * NS) {
         const int j = threadIdx.x >> 1;
         sh_span[threadIdx.x] = (probe && j < a.S) ? a.spans[((int64_t)s * a.S + j) * 2 + (threadIdx.x & 1)] : 0;
@@ -519,129 +527,157 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
             const int pos = min(first_pos[x] + row, L - 1);
             const float sl2 = a.scale_log2;
             float m_ref = -INFINITY, l = 0.f;
-            float sm[NS > 0 ? NS : 1];
-#pragma unroll
-            for (int js = 0; js < (NS > 0 ? NS : 1); ++js) sm[js] = 0.f;
+            // Span sums of the probe.  They live in shared memory (one column per thread, no bank conflicts)
+            // and not in registers: consecutive key tiles are almost always covered by the same set of spans,
+            // so their row sums collect in one running sum in a register, which is handed to the spans'
+            // accumulators only when the set changes; tiles with a span edge add their masked sums directly.
+            float* my_sm = &sh_sm[NS > 0 ? x : 0][0][NS > 0 ? row : 0];     // element of span j at my_sm[j * kBM]
+            if (NS > 0 && probe)
+                for (int js = 0; js < a.S; ++js) my_sm[js * kBM] = 0.f;
+            float run_acc = 0.f;
+            uint32_t run_mask = 0;
+            auto flush_run = [&]() {
+                for (uint32_t m = run_mask; m; m &= m - 1) my_sm[(__ffs(m) - 1) * kBM] += run_acc;
+                run_acc = 0.f;
+            };
 
-            for (int j = 0; j < nt && ok; ++j) {
-                ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), j & 1, abort_flag));
-                if (!ok) break;
-                tc_fence_after();
-                if (releases && (threadIdx.x & 127) == 0) {
-                    // QK(., j) has completed, and with it every MMA issued before it: K tile j and
-                    // V tile j - 1 are free for the producer
-                    mbar_arrive(smem_u32(&bars.k_empty[j & 1]));
-                    if (j > 0) mbar_arrive(smem_u32(&bars.v_empty[(j - 1) & 1]));
-                }
-                const int k0 = j * kBN;
-                const bool need_mask = (k0 + kBN - 1 > first_pos[x]);
+            // The key loop exists twice: heads without a probe run the plain loop, whatever the call probes
+            // elsewhere; probed heads carry the span sums.
+            auto key_loop = [&](auto probed_c) {
+                constexpr bool PROBED = decltype(probed_c)::value;
+                // spans touching a key tile: low byte covering, high byte straddling; looked up one tile ahead
+                auto tile_spans = [&](int j) -> uint32_t { return (j < kMaskTiles) ? sh_tile_mask[j] : classify_tile(sh_span, NS, j * kBN); };
+                uint32_t tm_next = PROBED ? tile_spans(0) : 0u;
+                for (int j = 0; j < nt && ok; ++j) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.s_full[x]), j & 1, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (releases && (threadIdx.x & 127) == 0) {
+                        // QK(., j) has completed, and with it every MMA issued before it: K tile j and
+                        // V tile j - 1 are free for the producer
+                        mbar_arrive(smem_u32(&bars.k_empty[j & 1]));
+                        if (j > 0) mbar_arrive(smem_u32(&bars.v_empty[(j - 1) & 1]));
+                    }
+                    const int k0 = j * kBN;
+                    const bool need_mask = (k0 + kBN - 1 > first_pos[x]);
 
-                uint32_t tm = 0;   // spans touching this key tile: low byte covering, high byte straddling
-                if (NS > 0 && probe) tm = (j < kMaskTiles) ? sh_tile_mask[j] : classify_tile(sh_span, NS, k0);
+                    const uint32_t tm = tm_next;
+                    if (PROBED && j + 1 < nt) tm_next = tile_spans(j + 1);
 
-                // the whole score row of this thread: four loads in flight, one wait
-                float sc[kBN];
+                    // the whole score row of this thread: four loads in flight, one wait
+                    float sc[kBN];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) tc_ld32(tS + 32 * c, sc + 32 * c);
+                    for (int c = 0; c < 4; ++c) tc_ld32(tS + 32 * c, sc + 32 * c);
 #pragma unroll
-                for (int c = 0; c < 4; ++c) tc_wait_ld_dep(sc + 32 * c);
-                if (need_mask) {
-                    // causal / end-of-sequence mask as a select (stale or poisoned keys never propagate)
-                    const int lim = pos - k0;
+                    for (int c = 0; c < 4; ++c) tc_wait_ld_dep(sc + 32 * c);
+                    if (need_mask) {
+                        // causal / end-of-sequence mask as a select (stale or poisoned keys never propagate)
+                        const int lim = pos - k0;
 #pragma unroll
-                    for (int i = 0; i < kBN; ++i) sc[i] = (i <= lim) ? sc[i] : -INFINITY;
-                }
-                float mxp[4];   // four independent chains keep the dependency depth short
+                        for (int i = 0; i < kBN; ++i) sc[i] = (i <= lim) ? sc[i] : -INFINITY;
+                    }
+                    float mxp[4];   // four independent chains keep the dependency depth short
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    float t = max3(sc[32 * q4], sc[32 * q4 + 1], sc[32 * q4 + 2]);
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        float t = max3(sc[32 * q4], sc[32 * q4 + 1], sc[32 * q4 + 2]);
 #pragma unroll
-                    for (int i = 3; i + 1 < 32; i += 2) t = max3(t, sc[32 * q4 + i], sc[32 * q4 + i + 1]);
-                    mxp[q4] = fmaxf(t, sc[32 * q4 + 31]);
-                }
-                const float mx = fmaxf(max3(mxp[0], mxp[1], mxp[2]), mxp[3]) * sl2;
+                        for (int i = 3; i + 1 < 32; i += 2) t = max3(t, sc[32 * q4 + i], sc[32 * q4 + i + 1]);
+                        mxp[q4] = fmaxf(t, sc[32 * q4 + 31]);
+                    }
+                    const float mx = fmaxf(max3(mxp[0], mxp[1], mxp[2]), mxp[3]) * sl2;
 
-                // raise the reference maximum only when it is exceeded by more than the threshold
-                const bool raise = mx > m_ref + kRescaleThreshold;
-                if (__any_sync(0xffffffffu, raise)) {
-                    const float m_new = fmaxf(m_ref, mx);
-                    const float f = (m_ref == -INFINITY) ? 0.f : fast_exp2(m_ref - m_new);
-                    m_ref = m_new;
-                    l *= f;
-#pragma unroll
-                    for (int js = 0; js < (NS > 0 ? NS : 1); ++js) sm[js] *= f;
-                    if (j > 0) {
-                        float v[32];
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            tc_ld32(tO + 32 * c, v);
-                            tc_wait_ld_dep(v);
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] *= f;
-                            tc_st32(tO + 32 * c, v);
+                    // raise the reference maximum only when it is exceeded by more than the threshold
+                    const bool raise = mx > m_ref + kRescaleThreshold;
+                    if (__any_sync(0xffffffffu, raise)) {
+                        const float m_new = fmaxf(m_ref, mx);
+                        const float f = (m_ref == -INFINITY) ? 0.f : fast_exp2(m_ref - m_new);
+                        m_ref = m_new;
+                        l *= f;
+                        if (PROBED) {
+                            run_acc *= f;
+                            for (int js = 0; js < a.S; ++js) my_sm[js * kBM] *= f;
                         }
-                        tc_wait_st();
+                        if (j > 0) {
+                            float v[32];
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                tc_ld32(tO + 32 * c, v);
+                                tc_wait_ld_dep(v);
+#pragma unroll
+                                for (int i = 0; i < 32; ++i) v[i] *= f;
+                                tc_st32(tO + 32 * c, v);
+                            }
+                            tc_wait_st();
+                        }
                     }
-                }
 
-                // probabilities in the frame of the reference maximum: fp32 for the sums, bf16 pairs
-                // written over the scores for the tensor cores
-                const float2 sl2v = make_float2(sl2, sl2), nmv = make_float2(-m_ref, -m_ref);
-                float2 rs2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                    // probabilities in the frame of the reference maximum: fp32 for the sums, bf16 pairs
+                    // written over the scores for the tensor cores
+                    const float2 sl2v = make_float2(sl2, sl2), nmv = make_float2(-m_ref, -m_ref);
+                    float2 rs2[4];   // row sums of the four 32-key chunks
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t pk[16];
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t pk[16];
+                        rs2[c] = make_float2(0.f, 0.f);
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int e = 32 * c + 2 * i;
-                        const float2 xx = __ffma2_rn(make_float2(sc[e], sc[e + 1]), sl2v, nmv);
-                        const float2 pp = make_float2(fast_exp2(xx.x), fast_exp2(xx.y));
-                        sc[e] = pp.x;
-                        sc[e + 1] = pp.y;
-                        rs2[i & 1] = __fadd2_rn(rs2[i & 1], pp);
-                        pk[i] = pack_bf16(pp.x, pp.y);
+                        for (int i = 0; i < 16; ++i) {
+                            const int e = 32 * c + 2 * i;
+                            const float2 xx = __ffma2_rn(make_float2(sc[e], sc[e + 1]), sl2v, nmv);
+                            const float2 pp = make_float2(fast_exp2(xx.x), fast_exp2(xx.y));
+                            if (PROBED) {   // kept for the masked sums of a tile with a span edge
+                                sc[e] = pp.x;
+                                sc[e + 1] = pp.y;
+                            }
+                            rs2[c] = __fadd2_rn(rs2[c], pp);
+                            pk[i] = pack_bf16(pp.x, pp.y);
+                        }
+                        tc_st16(tS + 16 * c, pk);
                     }
-                    tc_st16(tS + 16 * c, pk);
-                }
-                const float rs = (rs2[0].x + rs2[0].y) + (rs2[1].x + rs2[1].y);
-                l += rs;
-
-                // span masses: a tile inside a span adds the row sum, a straddling tile a masked sum
-                if (NS > 0 && probe) {
-                    if (tm & 0xffu) {
-#pragma unroll
-                        for (int js = 0; js < NS; ++js) sm[js] += ((tm >> js) & 1u) ? rs : 0.f;
-                    }
-                    if (tm & 0xff00u) {
+                    const float cs[4] = {rs2[0].x + rs2[0].y, rs2[1].x + rs2[1].y, rs2[2].x + rs2[2].y, rs2[3].x + rs2[3].y};
+                    const float rs = (cs[0] + cs[1]) + (cs[2] + cs[3]);
+                    l += rs;
+                    // P is complete: hand it to the MMA warp first, the span sums need registers only
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&bars.p_full[x]));
+                    if (PROBED) {
+                        // a tile inside spans adds its row sum to them (through the running sum)
+                        const uint32_t cover = tm & 0xffu;
+                        if (cover != run_mask) { flush_run(); run_mask = cover; }
+                        run_acc += rs;
+                        if (tm & 0xff00u) {
+                            // Spans with an edge inside the tile add prefix(hi) - prefix(lo), where prefix(t) is the
+                            // sum of the tile's first t probabilities: whole 32-key chunks from their row sums, the
+                            // chunk that holds the edge as a masked sum of the probabilities kept above.
+                            auto prefix = [&](int t) -> float {
+                                if (t <= 0) return 0.f;
+                                if (t >= kBN) return rs;
+                                const int c = t >> 5;
+                                const uint32_t r = (uint32_t)(t & 31);
+                                float acc[4] = {c > 0 ? cs[0] : 0.f, c > 1 ? cs[1] : 0.f, c > 2 ? cs[2] : 0.f, 0.f};
+#define HOOK_MASKED_CHUNK(C)                                                                        \
+    _Pragma("unroll") for (uint32_t i = 0; i < 32; ++i) acc[i & 3] += (i < r) ? sc[32 * (C) + i] : 0.f;
+                                switch (c) {   // static register indices in every case
+                                    case 0: HOOK_MASKED_CHUNK(0) break;
+                                    case 1: HOOK_MASKED_CHUNK(1) break;
+                                    case 2: HOOK_MASKED_CHUNK(2) break;
+                                    default: HOOK_MASKED_CHUNK(3) break;
+                                }
+#undef HOOK_MASKED_CHUNK
+                                return (acc[0] + acc[1]) + (acc[2] + acc[3]);
+                            };
 #pragma unroll 1
-                        for (int js = 0; js < NS; ++js) {
-                            if (!((tm >> (8 + js)) & 1u)) continue;
-                            const int lo = sh_span[2 * js] - k0, hi = sh_span[2 * js + 1] - k0;
-                            const uint32_t width = (uint32_t)(hi - lo);
-                            float acc0 = 0.f, acc1 = 0.f;
-#pragma unroll
-                            for (int i = 0; i < kBN; i += 2) {
-                                acc0 += ((uint32_t)(i - lo) < width) ? sc[i] : 0.f;
-                                acc1 += ((uint32_t)(i + 1 - lo) < width) ? sc[i + 1] : 0.f;
-                            }
-                            const float add = acc0 + acc1;
-                            switch (js) {   // static register targets
-                                case 0: sm[0] += add; break;
-                                case 1: if (NS > 1) sm[NS > 1 ? 1 : 0] += add; break;
-                                case 2: if (NS > 2) sm[NS > 2 ? 2 : 0] += add; break;
-                                case 3: if (NS > 3) sm[NS > 3 ? 3 : 0] += add; break;
-                                case 4: if (NS > 4) sm[NS > 4 ? 4 : 0] += add; break;
-                                case 5: if (NS > 5) sm[NS > 5 ? 5 : 0] += add; break;
-                                case 6: if (NS > 6) sm[NS > 6 ? 6 : 0] += add; break;
-                                default: if (NS > 7) sm[NS > 7 ? 7 : 0] += add; break;
+                            for (int js = 0; js < a.S; ++js) {
+                                if (!((tm >> (8 + js)) & 1u)) continue;
+                                my_sm[js * kBM] += prefix(sh_span[2 * js + 1] - k0) - prefix(sh_span[2 * js] - k0);
                             }
                         }
                     }
                 }
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(smem_u32(&bars.p_full[x]));
-            }
+                if (PROBED) flush_run();
+            };
+            if (NS > 0 && probe) key_loop(ProbedTag<true>{});
+            else key_loop(ProbedTag<false>{});
 
             // ---- epilogue: normalise, steer, round once, store ----
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.o_full[x]), 0, abort_flag));
@@ -651,7 +687,6 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
             if (ok) {
                 tc_fence_after();
                 const float al = hc.alpha[h];
-                const float* sv = a.steer + (int64_t)h * kHD;
                 // A thread holds one output row; stored from here, a warp would write 32 rows with 16
                 // bytes each per instruction.  The tile goes through the shared memory of Q_x instead
                 // (free: every MMA of this tile has completed), 16-byte chunks XOR-ed with the row so
@@ -668,7 +703,7 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
                         for (int i = 0; i < 4; ++i) {
                             const int d = 32 * c + 8 * q4 + 2 * i;
                             float y0 = v[8 * q4 + 2 * i] * inv, y1 = v[8 * q4 + 2 * i + 1] * inv;
-                            if (al != 0.f) { y0 = fmaf(al, sv[d], y0); y1 = fmaf(al, sv[d + 1], y1); }
+                            if (al != 0.f) { y0 += sh_steer[d]; y1 += sh_steer[d + 1]; }
                             w[i] = pack_bf16(y0, y1);
                         }
                         const uint32_t addr = stage + row * 256 + (((4 * c + q4) ^ (row & 7)) << 4);
@@ -698,9 +733,7 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
                     if (!last_only || row0[x] + row == n - 1) {
                         const int64_t mrow = last_only ? (int64_t)s : grow_seq + row0[x] + row;
                         float* dst = a.mass + (mrow * a.P + slot) * a.S;
-#pragma unroll
-                        for (int js = 0; js < NS; ++js)
-                            if (js < a.S) dst[js] = sm[js] * inv;
+                        for (int js = 0; js < a.S; ++js) dst[js] = my_sm[js * kBM] * inv;
                     }
                 }
             }
