@@ -248,7 +248,7 @@ struct ProbedTag {
 struct Barriers {
     uint64_t q_full[2];
     uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t s_full[2], p_half[2], p_full[2], o_full[2];   // p_half: the first 64 keys of P are in tensor memory
     uint64_t v_tail;          // the producer has zeroed the value rows past the end of the sequence
     uint32_t tmem_base;
     int abort_flag;
@@ -344,6 +344,7 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
         for (int x = 0; x < 2; ++x) {
             mbar_init(smem_u32(&bars.q_full[x]), 1);
             mbar_init(smem_u32(&bars.s_full[x]), 1);
+            mbar_init(smem_u32(&bars.p_half[x]), 128);
             mbar_init(smem_u32(&bars.p_full[x]), 128);
             mbar_init(smem_u32(&bars.o_full[x]), 1);
         }
@@ -468,11 +469,15 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
             }
             tc_commit(smem_u32(&bars.s_full[x]));
         };
-        auto issue_pv = [&](int x, int j) {
+        // P V in two halves of 64 keys each: the first half starts as soon as its probabilities are in tensor
+        // memory, while the softmax threads still work on the second
+        auto issue_pv_half = [&](int x, int j, int half) {
             const uint64_t dv = (j & 1) ? dV[1] : dV[0];
 #pragma unroll
-            for (int ks = 0; ks < kBN / 16; ++ks)
+            for (int kk = 0; kk < kBN / 32; ++kk) {
+                const int ks = half * (kBN / 32) + kk;
                 tc_mma_ts(tO[x], tS[x] + ks * 8, desc_advance(dv, (ks * 16 * 128) >> 4), idesc_pv, (ks > 0) || (j > 0));
+            }
         };
         // The whole warp walks the issue loop in step -- every lane looks at the barriers, so loop counters,
         // descriptors and branch conditions stay warp-uniform -- and one elected lane issues the MMAs and
@@ -501,11 +506,15 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
                 if (ok && j < ntiles[x]) {
+                    ok = mbar_wait(smem_u32(&bars.p_half[x]), j & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (elected) issue_pv_half(x, j, 0);
                     ok = mbar_wait(smem_u32(&bars.p_full[x]), j & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     if (elected) {
-                        issue_pv(x, j);
+                        issue_pv_half(x, j, 1);
                         if (j + 1 < ntiles[x]) issue_qk(x, j + 1);
                         else tc_commit(smem_u32(&bars.o_full[x]));
                     }
@@ -632,6 +641,11 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
                             pk[i] = pack_bf16(pp.x, pp.y);
                         }
                         tc_st16(tS + 16 * c, pk);
+                        if (c == 1) {   // the first 64 keys: the MMA warp may start on them
+                            tc_wait_st();
+                            tc_fence_before();
+                            mbar_arrive(smem_u32(&bars.p_half[x]));
+                        }
                     }
                     const float cs[4] = {rs2[0].x + rs2[0].y, rs2[1].x + rs2[1].y, rs2[2].x + rs2[2].y, rs2[3].x + rs2[3].y};
                     const float rs = (cs[0] + cs[1]) + (cs[2] + cs[3]);
