@@ -64,7 +64,7 @@ WORKLOADS = {
     # profiling sizes and the companions of the attention path (only with --workload)
     "cfg3_prefill": "prefill: 8 seqs x 4096 tokens causal, Hq32/Hkv8, D128, layer-0 probes, 3 spans, one layer call per step",
     "cfg3_prefill_small": "prefill, profiling size: 2 seqs x 2048 tokens causal, Hq32/Hkv8, D128, layer-0 probes, 3 spans",
-    "cfg5_decode_small": "long-context decode, profiling size: 4 seqs at 8192 keys, Hq64/Hkv8, D128, 64 probed heads, 8 spans",
+    "cfg5_decode_small": "long-context decode, profiling size: 4 seqs at 16384 keys, Hq64/Hkv8, D128, 64 probed heads, 8 spans",
     "steer_residual": "residual-stream steering: hidden[32768 x 4096] bf16 += alpha * vec, in place",
     "capture_qk": "raw q/k capture of the 16 probed heads of the decode batch (64 seqs, ctx U[512,4096])",
 }
@@ -73,7 +73,20 @@ TABLE = ["cfg2_decode", "cfg3_prefill_32layers", "cfg4_decode", "cfg4_prefill", 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the ncu captures
 # summarised under profiles/ (absent = no capture of the current kernel exists: reported as null).
-DRAM_TRAFFIC = {}
+DRAM_TRAFFIC = {
+    # hooked kernel of each workload, per launch
+    "cfg5_prefill": 18038.2e6,             # prefill_tc_kernel<8>, 64 x 516 CTAs
+    "cfg5_decode": 538.5e6,                # decode_stream_kernel<128,8>
+    "cfg5_decode_small": 268.8e6,
+    "cfg2_decode": 627.5e6,                # decode_splitk_kernel<128,2>
+    "cfg4_decode": 2515.9e6,               # decode_splitk_kernel<128,4>
+    "cfg4_prefill": 58.4e6,                # prefill_tc_kernel<8>, 28 x 18 CTAs
+    "cfg4_mixed": 2648.4e6,                # mixed_kernel<8,8>
+    "cfg3_prefill": 640.6e6,               # prefill_tc_kernel<8>, 32 x 136 CTAs
+    "cfg3_prefill_32layers": 32 * 640.6e6, # the same launch, 32 per step
+    "cfg3_prefill_small": 53.2e6,
+    "capture_qk": 841.0e6,                 # capture_k_kernel<128>
+}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -375,7 +388,7 @@ def build(ctx, name, binding):
     if name == "cfg4_mixed":
         return build_mixed(ctx, binding)
     if name == "cfg5_decode_small":
-        return build_single(ctx, inputs.config5_decode(tokens=8192, step=0, device=dev), binding)
+        return build_single(ctx, inputs.config5_decode(tokens=16384, step=0, device=dev), binding)
     raise SystemExit(f"unknown workload {name}; choose from {sorted(WORKLOADS)}")
 
 
@@ -642,8 +655,18 @@ def run_headline(args):
     sampler.start()
     windows, table = {}, {}
 
-    # ---- the headline: the long-context session, hooks on and off ----
+    # ---- the HBM-bound workloads first: a decode step runs some 100 us, and what the board does in the seconds
+    #      before (the long tensor-bound workloads drive it to its power cap) would otherwise be part of their numbers
     sess = Session(ctx, binding, probed=64)
+    if not dist and not args.headline_only:
+        table["cfg5_decode"], _ = measure_entry(ctx, "cfg5_decode", session_part(sess, "cfg5_decode"), warmup, windows)
+        for name in ("cfg2_decode", "cfg4_decode"):
+            w = build(ctx, name, binding)
+            table[name], _ = measure_entry(ctx, name, w, warmup, windows)
+            del w
+            torch.cuda.empty_cache()
+
+    # ---- the headline: the long-context session, hooks on and off ----
     head, th = measure_entry(ctx, HEADLINE, sess.entry(), warmup, windows, steps_per_block=spb, blocks=blocks, sync=barrier)
     barrier()
     t_step = sum(th) / len(th)                                 # mean over exactly `steps` timed steps
@@ -698,17 +721,16 @@ def run_headline(args):
 
     t_step, t_e2e = replicas.max_over_ranks([t_step, t_e2e], torch.device("cuda", local))
 
-    # ---- every other named workload (one GPU only: they are single-GPU measurements) ----
+    # ---- the tensor-bound workloads and the mixed step (one GPU only: they are single-GPU measurements) ----
     if not dist and not args.headline_only:
         table["cfg5_prefill"], _ = measure_entry(ctx, "cfg5_prefill", session_part(sess, "cfg5_prefill"), warmup, windows)
-        table["cfg5_decode"], _ = measure_entry(ctx, "cfg5_decode", session_part(sess, "cfg5_decode"), warmup, windows)
         del sess
         torch.cuda.empty_cache()
         s16 = Session(ctx, binding, probed=16)
         table["cfg5_16of64"], _ = measure_entry(ctx, "cfg5_16of64", s16.entry(), warmup, windows)
         del s16
         torch.cuda.empty_cache()
-        for name in ("cfg2_decode", "cfg4_decode", "cfg4_prefill", "cfg4_mixed", "cfg3_prefill_32layers"):
+        for name in ("cfg4_prefill", "cfg4_mixed", "cfg3_prefill_32layers"):
             w = build(ctx, name, binding)
             table[name], _ = measure_entry(ctx, name, w, warmup, windows)
             del w
@@ -727,7 +749,8 @@ def run_headline(args):
             "config": {"workload": f"{HEADLINE}: {WORKLOADS[HEADLINE]}",
                        "l2": "inputs larger than L2 (2.7 GB of q/K/V per prefill call, 0.54 GB of K/V per decode step)",
                        "replicas": world, "kv_cache": "resident in HBM (state, not a per-step input)",
-                       "inputs": "drawn on the device by a seeded generator (same recipe as the CPU-drawn test inputs)"},
+                       "inputs": "drawn on the device by a seeded generator (same recipe as the CPU-drawn test inputs)",
+                       "order": "HBM-bound table entries (decode) are timed before the headline, tensor-bound ones after it"},
             "roofline": roof, "hook_overhead": head["hook_overhead"], "ms_per_step_hooks_off": head["ms_per_step_hooks_off"],
             "prefill_ms": head["prefill_ms"], "decode_ms_per_step": head["decode_ms_per_step"], "decode_gbs": head["decode_gbs"],
             "e2e": {"value": replicas.replica_throughput(head["tokens_per_step"], t_e2e, world), "unit": UNIT,
