@@ -11,20 +11,26 @@
 //   warp  8    producer: resolves pages through the block table and issues one TMA box load per
 //              (page, 64-wide half of the head) into 128B-swizzled K and V stages; it also zeroes the
 //              value rows past the end of the sequence in the last tile;
-//   warp  9    owns tensor memory and walks the issue loop as a whole; one elected lane of it issues the MMAs: S = Q K^T (both operands
-//              K-major in shared memory) and O += P V (P from tensor memory, V as the MN-major B
-//              operand), ordered PV(A,j) QK(A,j+1) PV(B,j) QK(B,j+1) so that one tile's softmax
-//              overlaps the other tile's tensor work.  That thread is the pacemaker of the CTA, so
-//              it does nothing else: the K/V stages are handed back to the producer by a softmax
-//              thread of the later tile, which sees the completion of QK(.,j) anyway.
+//   warp  9    owns tensor memory and walks the issue loop as a whole, converged; one elected lane
+//              of it issues the MMAs: S = Q K^T (both operands K-major in shared memory) and
+//              O += P V (P from tensor memory, V as the MN-major B operand), ordered
+//              PV(A,j) QK(A,j+1) PV(B,j) QK(B,j+1) so that one tile's softmax overlaps the other
+//              tile's tensor work.  The pipe's queue of issued MMAs is shallow, so every cycle this
+//              warp spends on anything else is a cycle the pipe may run dry: it does nothing but
+//              wait and issue, the K/V stages are handed back to the producer by a softmax thread
+//              of the later tile (which sees the completion of QK(.,j) anyway), and P V of a tile
+//              is issued in two halves of 64 keys, the first as soon as the softmax has stored it.
 // Tensor memory (512 columns): S_A/P_A at 0, S_B/P_B at 128, O_A at 256, O_B at 384.
 //
 // The softmax keeps a *reference* maximum that is only raised when a tile's maximum exceeds it by
 // more than 2^8; probabilities, the running sum and the span accumulators all live in that frame,
 // so the result is exact (the reference cancels in o / l and s_j / l) while most tiles need no
 // rescale of the accumulator.  Span masses are added from the fp32 probabilities, before the
-// rounding to bf16: a key tile inside a span adds the tile's row sum, a tile that straddles a span
-// edge adds a masked row sum, a disjoint tile adds nothing.
+// rounding to bf16: a key tile inside a span adds its row sum to a running sum kept per set of
+// covering spans (flushed to the per-span sums, which live in shared memory, when the set changes);
+// a tile that straddles a span edge adds sums of the 32-key chunks inside the span plus a masked
+// sum of the one or two chunks on an edge; a disjoint tile adds nothing.  The probabilities are
+// handed to the MMA warp before any of this span work starts.
 //
 // Every wait on an mbarrier is bounded; when one runs out the role raises the CTA's abort flag (every
 // other wait of the CTA polls it and gives up too), the CTA reports HOOK_ATTN_ERR_TIMEOUT through the
