@@ -17,9 +17,10 @@
 //              PV(A,j) QK(A,j+1) PV(B,j) QK(B,j+1) so that one tile's softmax overlaps the other
 //              tile's tensor work.  The pipe's queue of issued MMAs is shallow, so every cycle this
 //              warp spends on anything else is a cycle the pipe may run dry: it does nothing but
-//              wait and issue, the K/V stages are handed back to the producer by a softmax thread
-//              of the later tile (which sees the completion of QK(.,j) anyway), and P V of a tile
-//              is issued in two halves of 64 keys, the first as soon as the softmax has stored it.
+//              wait and issue (plus one commit per step that hands the V stage back to the producer
+//              as soon as the step's last P V has completed; the K stage is handed back by a softmax
+//              thread of the later tile, which sees the completion of QK(.,j) anyway), and P V of a
+//              tile is issued in two halves of 64 keys, the first as soon as the softmax has stored it.
 // Tensor memory (512 columns): S_A/P_A at 0, S_B/P_B at 128, O_A at 256, O_B at 384.
 //
 // The softmax keeps a *reference* maximum that is only raised when a tile's maximum exceeds it by
@@ -521,6 +522,8 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
                     tc_fence_after();
                     if (elected) {
                         issue_pv_half(x, j, 1);
+                        // the step's last P V: once it has completed, V tile j is free for the producer
+                        if (x == 1 || j >= ntiles[1]) tc_commit(smem_u32(&bars.v_empty[st]));
                         if (j + 1 < ntiles[x]) issue_qk(x, j + 1);
                         else tc_commit(smem_u32(&bars.o_full[x]));
                     }
@@ -568,10 +571,9 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
                     if (!ok) break;
                     tc_fence_after();
                     if (releases && (threadIdx.x & 127) == 0) {
-                        // QK(., j) has completed, and with it every MMA issued before it: K tile j and
-                        // V tile j - 1 are free for the producer
+                        // QK(., j) has completed, and with it every MMA issued before it: K tile j is free for
+                        // the producer (V tiles are handed back by a commit of the MMA warp, which comes earlier)
                         mbar_arrive(smem_u32(&bars.k_empty[j & 1]));
-                        if (j > 0) mbar_arrive(smem_u32(&bars.v_empty[(j - 1) & 1]));
                     }
                     const int k0 = j * kBN;
                     const bool need_mask = (k0 + kBN - 1 > first_pos[x]);
