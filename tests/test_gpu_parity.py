@@ -521,6 +521,28 @@ def _random_case(seed, alpha_span):
                             poison=True, scale=None if ri(0, 1) else 0.05 + 0.1 * ri(0, 3))
 
 
+@pytest.mark.parametrize("probed", [False, True])
+def test_prefill_scores_that_keep_growing_along_the_keys(eng, probed):
+    """Keys whose scores climb in stairs along the sequence, with steps of 4, 16 and 49 (in log2 units) at
+    seeded positions: the running reference of the online softmax has to move again and again, in first and in
+    second halves of key tiles, on small steps that only add up and on steps that would overflow an
+    exponential taken against the old reference.  Every row and head is compared with the oracle."""
+    lens = [1000, 777, 300]
+    Hq, Hkv, D = 4, 2, 128
+    g = inputs._gen(77)
+    case = inputs.make_case("stairs", is_decode=False, seq_lens=lens, q_lens=lens, num_q_heads=Hq, num_kv_heads=Hkv,
+                            head_dim=D, seed=31, num_spans=3 if probed else 0,
+                            head_mask=torch.ones(Hq, dtype=torch.uint8) if probed else None, poison=True)
+    case.q[:] = 1.0                                   # score of key t = 128 * scale * k_val[t] = 11.3 k_val[t] (16.3 in log2)
+    for s, L in enumerate(lens):
+        steps = torch.tensor([0.0, 0.0, 0.0, 0.25, 1.0, 3.0])[torch.randint(0, 6, (L,), generator=g)]
+        steps[torch.rand(L, generator=g) > 0.03] = 0.0            # a stair every 30 keys or so
+        k_val = torch.cumsum(steps, 0).clamp(max=60.0)            # multiples of 0.25 up to 60: exact in bf16
+        for t in range(L):
+            case.k_cache[case.block_table[s, t // 16].item(), t % 16] = k_val[t].to(torch.bfloat16)
+    check(eng, case)
+
+
 @pytest.mark.parametrize("seed", range(24))
 def test_random_shapes_sweep(eng, seed):
     """Seeded random batches against the oracle at the stated tolerances, everywhere.  The steering is kept
