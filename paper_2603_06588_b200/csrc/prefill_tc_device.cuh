@@ -281,13 +281,46 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int kvh = h / a.G;
 
+    // The loads a CTA needs before it can start anything are issued side by side, not one after the other: a
+    // CTA lives for a few dozen microseconds, and every dependent trip to global memory at its start is half a
+    // microsecond in which its SM does nothing.
+    const volatile LaunchAbort* ab = &g_launch_abort;
+    const unsigned int ab_id = ab->launch_id;
+    const unsigned long long ab_when = ab->when_ns;
+
     // ---- locate (sequence, pair of query tiles); later pairs of a sequence (more keys) come first ----
-    int t = pair_index, s = 0, n = 0;
-    for (; s < a.num_seqs; ++s) {
-        n = a.cu_q_lens[s + 1] - a.cu_q_lens[s];
-        const int np = (n + 2 * kBM - 1) / (2 * kBM);
-        if (t < np) { t = np - 1 - t; break; }
-        t -= np;
+    // Every warp scans the sequences 32 at a time: a lane loads the row range and the length of its sequence, a
+    // prefix sum over the lanes' pair counts finds the sequence that holds pair `pair_index`.
+    int t = pair_index, s = -1, n = 0, L = 0;
+    int64_t grow_seq = 0;
+    for (int base = 0; base < a.num_seqs; base += 32) {
+        const int sq = base + lane;
+        int c0 = 0, c1 = 0, len = 0;
+        if (sq < a.num_seqs) {
+            c0 = a.cu_q_lens[sq];
+            c1 = a.cu_q_lens[sq + 1];
+            len = a.seq_lens[sq];
+        }
+        const int np = max(0, (c1 - c0 + 2 * kBM - 1) / (2 * kBM));
+        int incl = np;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        if (t < total) {
+            const int src = __ffs(__ballot_sync(0xffffffffu, t < incl)) - 1;   // first lane whose range ends past t
+            const int before = __shfl_sync(0xffffffffu, incl - np, src);
+            const int npair = __shfl_sync(0xffffffffu, np, src);
+            s = base + src;
+            n = __shfl_sync(0xffffffffu, c1 - c0, src);
+            L = __shfl_sync(0xffffffffu, len, src);
+            grow_seq = __shfl_sync(0xffffffffu, c0, src);
+            t = npair - 1 - (t - before);
+            break;
+        }
+        t -= total;
     }
     // last-token mode: a sequence without rows in this call gets zeros in its span_mass row
     if (NS > 0 && h == 0 && pair_index == 0 && a.probe_rows == HOOK_PROBE_ROWS_LAST) {
@@ -297,17 +330,12 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
             for (int i = lane; i < per; i += 32) a.mass[(int64_t)sq * per + i] = 0.f;
         }
     }
-    if (s >= a.num_seqs) return;
+    if (s < 0) return;
     // once any CTA of this launch has given up on a wait, the rest of the grid does not start
-    {
-        const volatile LaunchAbort* ab = &g_launch_abort;
-        if (ab->launch_id == launch_id && global_timer_ns() - ab->when_ns < kAbortWindowNs) {
-            if (threadIdx.x == 0) report(a.status, HOOK_ATTN_ERR_TIMEOUT);
-            return;
-        }
+    if (ab_id == launch_id && global_timer_ns() - ab_when < kAbortWindowNs) {
+        if (threadIdx.x == 0) report(a.status, HOOK_ATTN_ERR_TIMEOUT);
+        return;
     }
-    const int L = a.seq_lens[s];
-    const int64_t grow_seq = a.cu_q_lens[s];
     const int row0[2] = {2 * t * kBM, (2 * t + 1) * kBM};
     int rows[2], first_pos[2], ntiles[2];
 #pragma unroll
