@@ -803,7 +803,7 @@ def run_headline(args):
             "clocks": sampler.window(*windows[HEADLINE]),
             "workloads": table,
         }
-        if not args.no_cpu_baseline:
+        if not args.no_cpu_baseline and world == 1:     # the oracle is timed at N = 1 only
             cases = inputs.config5_session(device=dev)
             val, dt, desc, cores = run_oracle_sample(cases, budget_s=8.0, reps=2)
             line["cpu_baseline"] = dict({"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
