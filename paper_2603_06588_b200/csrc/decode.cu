@@ -51,6 +51,9 @@ __global__ void __launch_bounds__(kDecWarps * 32) decode_splitk_kernel(const Ker
     const int warp = threadIdx.x >> 5;
     const int G = a.G;
 
+    // launched with programmatic serialization: the merge of the call before this one on the stream may still be
+    // running (it reads the workspace this grid writes, and may be writing the q this grid reads)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int L = a.seq_lens[s];
     if (L <= 0 || L > a.max_keys) return;   // reported and zero-filled by the merge kernel
     const int start = c * a.chunk;
@@ -95,6 +98,9 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) decode_merge_kernel(const
     const int slot = hc.slot[h];
     float* mrow = (slot >= 0 && a.S > 0) ? a.mass + ((int64_t)s * a.P + slot) * a.S : nullptr;
 
+    // the first-stage kernel of the next call on the stream may be scheduled from here on: it waits for this grid
+    // before it touches the workspace or q
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // the partials are written by the kernel launched just before on the same stream
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
@@ -261,16 +267,31 @@ static cudaError_t launch_decode_t(KernelArgs a, const HeadCfg& hc, int num_sms,
     a.chunk = plan.chunk;
     a.max_chunks = plan.max_chunks;
     long parts;   // partials per unit, to size the merge block
+    // Programmatic serialization for the first kernel of the fixed-chunk cut as well: back-to-back decode calls on a
+    // stream overlap its launch with the merge of the call before (which releases its successor at once): decode
+    // batch 104.8 -> 102.3 us, mixed-batch decode 389.6 -> 384.2 us.  The one-wave streaming grid is launched in
+    // stream order: with the attribute its step got slower (94.8 -> 100.2 us with hooks, 92.7 -> 94.0 without).
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kDecWarps * 32);
+    cfg.dynamicSmemBytes = decode_smem_bytes<HD>();
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = plan.stream ? 0 : 1;
+    cudaError_t e;
     if (plan.stream) {
         const int ctas = kDecCtasPerSM * (num_sms < kDecMaxSMs ? (num_sms > 0 ? num_sms : 1) : kDecMaxSMs);
         a.workers = ctas * kDecWarps;
-        decode_stream_kernel<HD, NS><<<ctas, kDecWarps * 32, decode_smem_bytes<HD>(), st>>>(a, hc);
+        cfg.gridDim = dim3(ctas);
+        e = cudaLaunchKernelEx(&cfg, decode_stream_kernel<HD, NS>, a, hc);
         parts = stream_parts_estimate(a, ctas, kDecWarps);
     } else {
-        decode_splitk_kernel<HD, NS><<<dim3(plan.max_chunks, a.Hkv, a.num_seqs), kDecWarps * 32, decode_smem_bytes<HD>(), st>>>(a, hc);
+        cfg.gridDim = dim3(plan.max_chunks, a.Hkv, a.num_seqs);
+        e = cudaLaunchKernelEx(&cfg, decode_splitk_kernel<HD, NS>, a, hc);
         parts = plan.max_chunks;
     }
-    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return launch_merge<HD>(a, hc, plan.stream, parts, st);
 }

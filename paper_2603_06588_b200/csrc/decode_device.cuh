@@ -394,6 +394,11 @@ __device__ __forceinline__ void decode_stream_cta(const KernelArgs& a, const Hea
     __syncthreads();
     // the merge kernel may be scheduled from here on; it waits for this grid's writes itself
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // Launched with programmatic serialization, this grid may have started while the merge of the call before it
+    // on the stream was still running (that merge lets its successor go at once); everything up to here read the
+    // sequence lengths only.  From here on the grid writes the workspace, which that merge may be reading, and reads
+    // q, which may be what that merge wrote: wait for it.  (Without such a predecessor the wait returns at once.)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (cta == 0) {   // the merge kernel sizes up its unit from this table
         int* prefix = reinterpret_cast<int*>(a.ws);
         for (int i = threadIdx.x; i < a.num_seqs; i += NT) prefix[i] = sh_ex[i];
