@@ -76,12 +76,12 @@ TABLE = ["cfg2_decode", "cfg3_prefill_32layers", "cfg4_decode", "cfg4_prefill", 
 DRAM_TRAFFIC = {
     # hooked kernel of each workload, per launch
     "cfg5_prefill": 18028.9e6,             # prefill_tc_kernel<8>, 64 x 516 CTAs
-    "cfg5_decode": 538.5e6,                # decode_stream_kernel<128,8>
+    "cfg5_decode": 538.4e6,                # decode_stream_kernel<128,8>
     "cfg5_decode_small": 268.8e6,
-    "cfg2_decode": 627.5e6,                # decode_splitk_kernel<128,2>
-    "cfg4_decode": 2515.9e6,               # decode_splitk_kernel<128,4>
+    "cfg2_decode": 627.7e6,                # decode_splitk_kernel<128,2>
+    "cfg4_decode": 2515.8e6,               # decode_splitk_kernel<128,4>
     "cfg4_prefill": 58.1e6,                # prefill_tc_kernel<8>, 28 x 18 CTAs
-    "cfg4_mixed": 2651.2e6,                # mixed_kernel<8,8>
+    "cfg4_mixed": 2651.1e6,                # mixed_kernel<8,8>
     "cfg3_prefill": 640.5e6,               # prefill_tc_kernel<8>, 32 x 136 CTAs
     "cfg3_prefill_32layers": 32 * 640.5e6, # the same launch, 32 per step
     "cfg3_prefill_small": 53.2e6,
