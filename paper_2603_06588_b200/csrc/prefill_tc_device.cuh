@@ -458,9 +458,6 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
     // Register split between the warpgroups: the softmax threads keep a whole 128-wide score row in
     // registers, the producer/MMA warpgroup needs few.  Launched with 168 per thread (384 x 168 =
     // 64512); after the split 128 x (208 + 208 + 72) = 62464, which fits the launch allocation.
-
-
-
     if (warp >= 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 72;" ::: "memory");
     }
@@ -470,7 +467,7 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
         if (ok && nmax > 0 && nmax * kBN > L) {
             // value rows at keys >= L (page tails, pages that were never loaded) must not reach the
             // tensor cores: 0 * NaN would poison the accumulator.  Zero them in shared memory once the
-            // last tile has landed, then tell the MMA thread.
+            // last tile has landed, then tell the MMA warp.
             const int j = nmax - 1, st = j & 1;
             ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1, abort_flag));
             if (ok) {
@@ -491,7 +488,7 @@ __device__ __forceinline__ void prefill_tc_cta(const KernelArgs& a, const HeadCf
         constexpr uint32_t idesc_qk = instr_desc(0), idesc_pv = instr_desc(1);
         const uint32_t tS[2] = {tmem, tmem + 128}, tO[2] = {tmem + 256, tmem + 384};
         // Descriptors are built once; per MMA only the start-address field moves (one 32-bit add), so
-        // that the single issuing thread keeps the tensor pipe fed.
+        // that the issuing lane keeps the tensor pipe fed.
         const uint64_t dQ[2] = {smem_desc(sQ[0], 16, 1024), smem_desc(sQ[1], 16, 1024)};
         const uint64_t dK[2] = {smem_desc(sK, 16, 1024), smem_desc(sK + kTileBytes, 16, 1024)};
         const uint64_t dV[2] = {smem_desc(sV, kHalfBytes, 1024), smem_desc(sV + kTileBytes, kHalfBytes, 1024)};
