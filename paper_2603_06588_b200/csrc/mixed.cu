@@ -62,7 +62,7 @@ cudaError_t configure_mixed()
 {
     cudaError_t e;
 #define HOOK_CFG(A, B) if ((e = cudaFuncSetAttribute(mixed_kernel<A, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes)) != cudaSuccess) return e;
-    HOOK_CFG(0, 0) HOOK_CFG(0, 8) HOOK_CFG(8, 0) HOOK_CFG(8, 8)
+    HOOK_CFG(0, 0) HOOK_CFG(0, 4) HOOK_CFG(0, 8) HOOK_CFG(8, 0) HOOK_CFG(8, 4) HOOK_CFG(8, 8)
 #undef HOOK_CFG
     return cudaSuccess;
 }
@@ -111,11 +111,16 @@ cudaError_t launch_mixed(const KernelArgs& apf, const HeadCfg& hpf, const Kernel
     const int dec_ctas = mixed_decode_ctas(apf, adec, num_sms, forced_dec_ctas);
     adec.workers = dec_ctas * kMixWarps;
     const long grid = (long)dec_ctas + (long)prefill_tc_pairs(apf) * apf.Hq;
-    const bool ppf = apf.any_probe, pdec = adec.any_probe;
+    // the prefill role has two forms (no spans, up to 8); the decode role keeps its span sums in registers and has
+    // one for up to 4 spans as well
+    const bool ppf = apf.any_probe;
+    const int nsd = !adec.any_probe ? 0 : (adec.S <= 4 ? 4 : 8);
     cudaError_t e;
-    if (ppf && pdec) e = launch_mixed_t<8, 8>(apf, hpf, adec, hdec, mq, mk, mv, dec_ctas, grid, st);
+    if (ppf && nsd == 8) e = launch_mixed_t<8, 8>(apf, hpf, adec, hdec, mq, mk, mv, dec_ctas, grid, st);
+    else if (ppf && nsd == 4) e = launch_mixed_t<8, 4>(apf, hpf, adec, hdec, mq, mk, mv, dec_ctas, grid, st);
     else if (ppf) e = launch_mixed_t<8, 0>(apf, hpf, adec, hdec, mq, mk, mv, dec_ctas, grid, st);
-    else if (pdec) e = launch_mixed_t<0, 8>(apf, hpf, adec, hdec, mq, mk, mv, dec_ctas, grid, st);
+    else if (nsd == 8) e = launch_mixed_t<0, 8>(apf, hpf, adec, hdec, mq, mk, mv, dec_ctas, grid, st);
+    else if (nsd == 4) e = launch_mixed_t<0, 4>(apf, hpf, adec, hdec, mq, mk, mv, dec_ctas, grid, st);
     else e = launch_mixed_t<0, 0>(apf, hpf, adec, hdec, mq, mk, mv, dec_ctas, grid, st);
     if (e != cudaSuccess) return e;
     return launch_decode_stream_merge(adec, hdec, dec_ctas, kMixWarps, st);

@@ -74,11 +74,12 @@ def _run_mixed(eng, pf, dec):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("dec_ctas", [0, 1, 37])
-def test_mixed_small_ragged_step_matches_the_oracle(dec_ctas, monkeypatch):
+@pytest.mark.parametrize("dec_ctas,spans_dec", [(0, 3), (1, 3), (37, 3), (0, 6), (0, 8)])
+def test_mixed_small_ragged_step_matches_the_oracle(dec_ctas, spans_dec, monkeypatch):
     """Ragged decode batch (a unit shared by many warps, warps that cross units, empty shares) next to chunked
     prefill with partial tiles; every row of both halves is checked.  Run with the split chosen from the
-    shapes, with a single decode CTA and with more decode CTAs than the batch has work for."""
+    shapes, with a single decode CTA and with more decode CTAs than the batch has work for, and with span counts
+    of the decode half on either side of the decode role's two probing forms (up to 4 spans, up to 8)."""
     if dec_ctas:
         monkeypatch.setenv("HOOK_ATTN_MIXED_DECODE_CTAS", str(dec_ctas))
     else:
@@ -91,7 +92,7 @@ def test_mixed_small_ragged_step_matches_the_oracle(dec_ctas, monkeypatch):
     alpha[2], alpha[5] = 0.8, -0.5
     mask = torch.tensor([1, 0, 0, 1, 1, 0, 1, 0], dtype=torch.uint8)
     dec = inputs.make_case("mix_dec", is_decode=True, seq_lens=lens, q_lens=[1] * len(lens), num_q_heads=8, num_kv_heads=2,
-                           head_dim=128, seed=92, num_spans=3, head_mask=mask, alpha=alpha, steer=True,
+                           head_dim=128, seed=92, num_spans=spans_dec, head_mask=mask, alpha=alpha, steer=True,
                            probe_rows=inputs.PROBE_ROWS_LAST, poison=True)
     pf = inputs.make_case("mix_pf", is_decode=False, seq_lens=[700, 300, 90, 260], q_lens=[200, 300, 0, 129], num_q_heads=8,
                           num_kv_heads=2, head_dim=128, seed=93, num_spans=3, head_mask=mask, alpha=alpha, steer=True,
