@@ -81,7 +81,7 @@ DRAM_TRAFFIC = {
     "cfg2_decode": 627.7e6,                # decode_splitk_kernel<128,2>
     "cfg4_decode": 2515.8e6,               # decode_splitk_kernel<128,4>
     "cfg4_prefill": 58.1e6,                # prefill_tc_kernel<8>, 28 x 18 CTAs
-    "cfg4_mixed": 2651.1e6,                # mixed_kernel<8,8>
+    "cfg4_mixed": 2649.0e6,                # mixed_kernel<8,4>
     "cfg3_prefill": 640.5e6,               # prefill_tc_kernel<8>, 32 x 136 CTAs
     "cfg3_prefill_32layers": 32 * 640.5e6, # the same launch, 32 per step
     "cfg3_prefill_small": 53.2e6,
