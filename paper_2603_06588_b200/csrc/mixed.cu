@@ -81,8 +81,8 @@ size_t mixed_decode_workspace_bytes(int num_seqs, int Hkv, int G, int head_dim)
 
 // How many CTAs take the decode role.  The host knows bounds, not lengths: the decode call is taken to read
 // 0.55 of the keys its bound allows and the prefill rows to see 0.8 of theirs.  An SM in the decode role is
-// taken to stream 60 GB/s (twelve warps with one 8 KB page in flight each; 75-90 GB/s were measured with
-// few decode SMs, less once HBM fills up), an SM in the prefill role to
+// taken to stream 60 GB/s (52 GB/s when it probes; twelve warps with one 8 KB page in flight each; 75-90 GB/s were
+// measured with few decode SMs, less once HBM fills up), an SM in the prefill role to
 // sustain 5.7 TFLOP/s; the split equalises the two times.  Too many decode CTAs cost little -- their SMs go to
 // prefill CTAs when they are done -- too few leave the decode as the long pole, so the result is rounded up.
 int mixed_decode_ctas(const KernelArgs& apf, const KernelArgs& adec, int num_sms, int forced)
@@ -93,7 +93,9 @@ int mixed_decode_ctas(const KernelArgs& apf, const KernelArgs& adec, int num_sms
     } else {
         const double bytes = 0.55 * (double)adec.num_seqs * adec.Hkv * adec.max_keys * 4.0 * 128;
         const double flops = 0.8 * (double)apf.total_q * apf.Hq * apf.max_keys * 4.0 * 128;
-        const double t_dec1 = bytes / 60e9, t_pf1 = flops / 5.7e12;     // seconds on one SM
+        // with span sums to carry, a decode SM streams less: measured optimum 72 CTAs against 64-67 without (0.585
+        // against 0.596 ms at 67)
+        const double t_dec1 = bytes / (adec.any_probe ? 52e9 : 60e9), t_pf1 = flops / 5.7e12;     // seconds on one SM
         d = (int)(num_sms * t_dec1 / (t_dec1 + t_pf1) + 0.999) + 2;
     }
     if (d > num_sms - 8) d = num_sms - 8;
