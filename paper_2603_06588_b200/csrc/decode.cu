@@ -101,10 +101,13 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) decode_merge_kernel(const
     // the first-stage kernel of the next call on the stream may be scheduled from here on: it waits for this grid
     // before it touches the workspace or q
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // what does not come from the first-stage kernel is fetched while that kernel still runs
+    const int L = a.seq_lens[s];
+    const float al = hc.alpha[h];
+    const float steer_d = (al != 0.f && (int)threadIdx.x < HD) ? al * a.steer[(int64_t)h * HD + threadIdx.x] : 0.f;
     // the partials are written by the kernel launched just before on the same stream
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    const int L = a.seq_lens[s];
     const int np = decode_pages(L, a.max_keys);
     if (np == 0) {
         if (threadIdx.x == 0) report(a.status, L <= 0 ? HOOK_ATTN_ERR_INVALID_ARG : HOOK_ATTN_ERR_BOUNDS);
@@ -197,9 +200,7 @@ __global__ void __launch_bounds__(kMergeMaxWarps * 32) decode_merge_kernel(const
     }
     const float inv = 1.f / ltot;
     if (d < HD) {
-        val *= inv;
-        const float al = hc.alpha[h];
-        if (al != 0.f) val += al * a.steer[(int64_t)h * HD + d];
+        val = val * inv + steer_d;
         orow[d] = __float2bfloat16(val);
     }
     if (mrow && d < a.S) mrow[d] = mm * inv;
